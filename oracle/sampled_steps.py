@@ -1,0 +1,233 @@
+"""The sampled selector restated step by step (test infrastructure only).
+
+Follows the paper's notation and order, one row at a time, with numpy:
+
+  Phase 1 (Section 4.2): coarse map c(x), row-phased stride-s view V_{r,s},
+          sample histogram h, inclusive prefix H, tau_0 = min{b : H(b) >= q},
+          nested tau_1 >= tau_0 from the same prefix.
+  Phase 2 (Section 4.3): admitted tail A(tau) = {i : c(x_i) <= tau}, its size
+          C(tau), the leading-digit histogram of kappa_32-descending; band
+          extension A(tau_1) \\ A(tau_0) on underfill; exact coarse recovery
+          (tau_star over the complete row) when the band is still short.
+  Phase 3 (Section 4.4): D = 3 radix rounds over digits of widths 11+11+10:
+          b_j = min{b : H_j(b) >= k_j}, commit digits < b_j, keep digit == b_j,
+          k_{j+1} = k_j - |R_j|; then fill the k_D remaining slots from the
+          final equal-key group.
+
+Readings where the paper leaves a choice open (all performance-only except the
+tie rule, which follows the operator definition used by this repository):
+
+* final equal-key group: the lowest indices are taken;
+* pi_s: bit reversal of (r mod s) over log2(s) bits;
+* stride per K: the largest power of two s <= 128 with s <= K/16 (so the primary
+  sample rank q = ceil(1.5 K / s) stays >= 24); s = 128 at K = 2048 as evaluated;
+* margins: K~ = 1.5 K, K~_1 = 1.75 K (Sections 4.2 and 6.4);
+* fp16 projection: IEEE round-to-nearest-even, overflow to inf, subnormals kept;
+  a NaN pattern (outside the contract) is placed by its sign: bin 0 if positive,
+  bin 2047 if negative, which keeps c monotone in the key order;
+* candidate capacity: max(4 K, 4096) entries; a row whose admitted tail exceeds
+  it is routed to recovery (the paper spills to global memory instead);
+* rows with K < L <= capacity skip Phase 1: everything is admitted (C = L) and
+  Phase 3 runs on the whole row ("direct" route).
+
+`select_row` returns the selected index set and a trace of the intermediate
+quantities; the set must equal the plain definition (Theorem "End-to-End
+Exactness"), which tests/ check on every input they use.
+"""
+from dataclasses import dataclass, field
+
+import numpy as np
+
+B_C = 2048                      # coarse bins, Eq. "coarse-map"
+DIGIT_WIDTHS = (11, 11, 10)     # Section 4.3, D = 3
+
+ROUTE_SHORT = 0      # L <= K: every index, then sentinels
+ROUTE_DIRECT = 1     # K < L <= capacity: admit all, Phase 3
+ROUTE_PRIMARY = 2    # C(tau_0) >= K
+ROUTE_BAND = 3       # C(tau_0) < K <= C(tau_1)
+ROUTE_RECOVERY = 4   # underfill after the band, or unusable view
+ROUTE_OVERFLOW = 5   # admitted tail larger than the candidate capacity
+ROUTE_NAMES = ("short", "direct", "primary", "band", "recovery", "overflow")
+
+
+def stride_for(K):
+    s = 1
+    while s * 2 <= 128 and (s * 2) * 16 <= K:
+        s *= 2
+    return s
+
+
+def capacity_for(K):
+    return max(4 * K, 4096)
+
+
+def sample_ranks(K, s):
+    """q = ceil(1.5 K / s), q_1 = ceil(1.75 K / s) in exact integer arithmetic."""
+    q = -(-3 * K // (2 * s))
+    q1 = -(-7 * K // (4 * s))
+    return q, q1
+
+
+def phase_offset(r, s):
+    """a_r = pi_s(r mod s) with pi_s = bit reversal over log2(s) bits."""
+    bits = s.bit_length() - 1
+    v = r % s
+    out = 0
+    for _ in range(bits):
+        out = (out << 1) | (v & 1)
+        v >>= 1
+    return out
+
+
+def kappa32_desc(x):
+    """Descending sortable key of the FP32 score: larger value, smaller key."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    neg = (u >> np.uint32(31)).astype(bool)
+    asc = np.where(neg, ~u, u | np.uint32(0x80000000)).astype(np.uint32)
+    return ~asc
+
+
+def coarse_bin(x):
+    """c(x) = floor(kappa_16-descending(fp16(x)) / 2^5), Eq. "coarse-map"."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    with np.errstate(over="ignore"):
+        h = x.astype(np.float16).view(np.uint16).astype(np.uint32)
+    neg = (h >> 15).astype(bool)
+    asc16 = np.where(neg, h ^ 0xFFFF, h | 0x8000)
+    c = ((0xFFFF - asc16) >> 5).astype(np.int64)
+    u = x.view(np.uint32)
+    is_nan = (u & np.uint32(0x7FFFFFFF)) > np.uint32(0x7F800000)
+    c = np.where(is_nan, np.where((u >> np.uint32(31)).astype(bool), B_C - 1, 0), c)
+    return c
+
+
+def digit(kappa, j):
+    """dig_j of a 32-bit descending key under the 11+11+10 split."""
+    shift = 32 - sum(DIGIT_WIDTHS[: j + 1])
+    return (kappa >> np.uint32(shift)) & np.uint32((1 << DIGIT_WIDTHS[j]) - 1)
+
+
+def first_reaching(hist, quota):
+    """min{b : H(b) >= quota} for the inclusive prefix H of ``hist``; -1 if none."""
+    H = np.cumsum(hist)
+    hit = np.nonzero(H >= quota)[0]
+    return int(hit[0]) if len(hit) else -1
+
+
+@dataclass
+class Trace:
+    route: int = -1
+    stride: int = 0
+    a_r: int = 0
+    n_view: int = 0
+    q: int = 0
+    q1: int = 0
+    tau0: int = -1
+    tau1: int = -1
+    C0: int = 0            # C(tau_0)
+    C1: int = 0            # C(tau_1) (0 unless the band was attempted)
+    tau_star: int = -1
+    frontier: list = field(default_factory=list)   # |Q_j| entering round j
+    quotas: list = field(default_factory=list)     # k_j entering round j
+    boundary_digits: list = field(default_factory=list)
+
+
+def refine(x, E0, Q0, k0, trace=None):
+    """Phase 3 on the interface tuple (E_0, Q_0, k_0); h_0 is rebuilt from Q_0."""
+    kappa = kappa32_desc(x)
+    E = list(E0)
+    Q = np.asarray(Q0, dtype=np.int64)
+    k = int(k0)
+    for j in range(len(DIGIT_WIDTHS)):
+        if trace is not None:
+            trace.frontier.append(len(Q))
+            trace.quotas.append(k)
+        if k == 0:
+            Q = Q[:0]
+            break
+        d = digit(kappa[Q], j).astype(np.int64)
+        h = np.bincount(d, minlength=1 << DIGIT_WIDTHS[j])
+        b = first_reaching(h, k)
+        assert b >= 0, "certified state must hold at least k_j indices"
+        if trace is not None:
+            trace.boundary_digits.append(b)
+        R = Q[d < b]
+        E.extend(R.tolist())
+        k -= len(R)
+        Q = Q[d == b]
+    # Q_D: identical keys; the lowest indices fill the remaining k_D slots.
+    E.extend(np.sort(Q)[:k].tolist())
+    return np.asarray(sorted(E), dtype=np.int32)
+
+
+def select_row(x, r, K, stride=None, capacity=None):
+    """Run the three phases on row ``r`` with valid scores ``x``.
+
+    Returns (indices ascending int32 array of length min(K, L), Trace).
+    """
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    L = len(x)
+    s = stride_for(K) if stride is None else stride
+    cap = capacity_for(K) if capacity is None else capacity
+    t = Trace(stride=s)
+    t.q, t.q1 = sample_ranks(K, s)
+    if L <= K:
+        t.route = ROUTE_SHORT
+        return np.arange(L, dtype=np.int32), t
+    every = np.arange(L, dtype=np.int64)
+    if L <= cap:
+        t.route = ROUTE_DIRECT
+        t.C0 = L
+        return refine(x, [], every, K, t), t
+
+    c = coarse_bin(x)
+
+    def exact_coarse_recovery():
+        h_all = np.bincount(c, minlength=B_C)
+        t.tau_star = first_reaching(h_all, K)
+        E0 = every[c < t.tau_star]
+        Q0 = every[c == t.tau_star]
+        return refine(x, E0.tolist(), Q0, K - len(E0), t)
+
+    # Phase 1
+    t.a_r = phase_offset(r, s)
+    view = np.arange(t.a_r, L, s, dtype=np.int64)
+    t.n_view = len(view)
+    if t.n_view < t.q1:
+        t.route = ROUTE_RECOVERY
+        return exact_coarse_recovery(), t
+    h = np.bincount(c[view], minlength=B_C)
+    t.tau0 = first_reaching(h, t.q)
+    t.tau1 = first_reaching(h, t.q1)
+
+    # Phase 2
+    A0 = every[c <= t.tau0]
+    t.C0 = len(A0)
+    if t.C0 > cap:
+        t.route = ROUTE_OVERFLOW
+        return exact_coarse_recovery(), t
+    if t.C0 >= K:
+        t.route = ROUTE_PRIMARY
+        return refine(x, [], A0, K, t), t
+    A1 = every[c <= t.tau1]
+    t.C1 = len(A1)
+    if t.C1 > cap:
+        t.route = ROUTE_OVERFLOW
+        return exact_coarse_recovery(), t
+    if t.C1 >= K:
+        t.route = ROUTE_BAND
+        return refine(x, [], A1, K, t), t
+    t.route = ROUTE_RECOVERY
+    return exact_coarse_recovery(), t
+
+
+def select_rows(scores, row_starts, row_lengths, K, stride=None, capacity=None):
+    """All rows of a packed batch; returns (list of index arrays, list of Trace)."""
+    sets, traces = [], []
+    for r in range(len(row_lengths)):
+        L = max(int(row_lengths[r]), 0)
+        s0 = int(row_starts[r])
+        idx, tr = select_row(scores[s0:s0 + L], r, K, stride, capacity)
+        sets.append(idx)
+        traces.append(tr)
+    return sets, traces
