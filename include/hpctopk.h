@@ -1,0 +1,132 @@
+/* hpctopk - exact Top-K selection over ragged FP32 score rows on NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library built from paper_2609_08450_b200/csrc/.  Unless a comment
+ * says "host", every pointer below is a DEVICE pointer owned by the caller.  The
+ * library allocates nothing and keeps no per-call state; the only process-wide
+ * state is a per-device cache of launch attributes filled on first use.
+ *
+ * The operation is the standalone selector of "Sample-Guided Exact Top-K Selection
+ * for Long-Context Sparse Attention": the operator contract of Section 2.1, computed
+ * with the three phases of Section 4 (coarse boundary from a fixed-stride sample,
+ * one fused complete-row certification/compaction pass, exact radix refinement of
+ * the frontier) plus the recovery routes of Section 4.3.
+ */
+#ifndef HPCTOPK_H_
+#define HPCTOPK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* A CUDA stream handle (cudaStream_t), spelled without the CUDA headers. */
+typedef struct CUstream_st* hpctopk_stream_t;
+
+typedef enum {
+  HPCTOPK_OK = 0,
+  HPCTOPK_ERR_INVALID_ARG = 1,   /* null pointer, negative count, K < 1 */
+  HPCTOPK_ERR_UNSUPPORTED_K = 2, /* K > HPCTOPK_MAX_K */
+  HPCTOPK_ERR_MISALIGNED = 3,    /* scores not 16-byte aligned, workspace not 256-byte aligned */
+  HPCTOPK_ERR_WORKSPACE = 4,     /* reserved */
+  HPCTOPK_ERR_CUDA = 5,          /* a CUDA runtime call failed (no device, launch error) */
+  HPCTOPK_ERR_TIMEOUT = 6        /* reserved: the kernels contain no waits */
+} hpctopk_status;
+
+#define HPCTOPK_MAX_K 4096
+
+/* How a row was resolved (Sections 4.2-4.3).  Values index hpctopk_stats.rows_by_route. */
+enum {
+  HPCTOPK_ROUTE_SHORT = 0,    /* L <= K: every valid index, then sentinels (Section 2.1) */
+  HPCTOPK_ROUTE_DIRECT = 1,   /* K < L <= capacity: whole row admitted, refined on chip */
+  HPCTOPK_ROUTE_PRIMARY = 2,  /* C(tau_0) >= K: certified by the primary boundary */
+  HPCTOPK_ROUTE_BAND = 3,     /* C(tau_0) < K <= C(tau_1): certified after the band extension */
+  HPCTOPK_ROUTE_RECOVERY = 4, /* still underfilled (or view unusable): full-radix exact recovery */
+  HPCTOPK_ROUTE_OVERFLOW = 5  /* admitted tail larger than the on-chip capacity: exact recovery */
+};
+
+/* Counters of the most recent hpctopk_select call on a workspace (host struct). */
+typedef struct {
+  uint64_t rows_by_route[6];  /* rows resolved by each HPCTOPK_ROUTE_* */
+  uint64_t rows_split;        /* rows whose complete-row pass was partitioned over several CTAs */
+  uint64_t tasks;             /* row or row-segment tasks executed */
+  uint64_t candidates_sum;    /* sum over sampled rows of C(tau) entering refinement */
+  uint64_t candidates_max;    /* max over sampled rows of the same */
+  uint64_t elements_sampled;  /* score reads issued by Phase 1 (all replicas) */
+  uint64_t elements_scanned;  /* score reads issued by complete-row passes (all routes) */
+  uint64_t elements_valid;    /* sum of valid row lengths */
+  uint64_t error_flags;       /* nonzero: an internal invariant was violated */
+  uint64_t reserved[2];
+} hpctopk_stats;
+
+/* Per-row record of the most recent call (host struct; see hpctopk_read_row_info). */
+typedef struct {
+  int32_t route;    /* HPCTOPK_ROUTE_* */
+  int32_t tau;      /* tau_0 | (tau_1 << 16) for sampled rows, -1 otherwise (Eq. "primary-threshold") */
+  int32_t c_tau0;   /* C(tau_0), Eq. "candidate-set"; L on the direct route */
+  int32_t c_final;  /* size of the admitted tail that entered refinement (0 on recovery/short) */
+} hpctopk_row_info;
+
+/* Library version, 1000*major + minor.  Host only; never fails. */
+int hpctopk_version(void);
+
+/* Text for a status code.  Host only; returns a static string. */
+const char* hpctopk_status_string(int status);
+
+/* Bytes of device workspace hpctopk_select needs for up to `max_num_rows` rows at rank K.
+ * Bounded by a constant plus 16 bytes per row (independent of row width; Section 2.1,
+ * "Deployment requirements").  Host only.  Returns 0 for invalid arguments. */
+size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K);
+
+/* Policy the selector applies at rank K to a row of valid length L (host mirror of the
+ * device-side routing; lets a caller build inputs that alias the sampling stride).
+ *   stride   <- s of the row-phased view V_{r,s} (Eq. "view")
+ *   capacity <- on-chip candidate capacity (entries)
+ *   route    <- HPCTOPK_ROUTE_SHORT, HPCTOPK_ROUTE_DIRECT, or HPCTOPK_ROUTE_PRIMARY meaning
+ *               "enters the sampled path"
+ * Any output pointer may be NULL.  Host only. */
+int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route);
+
+/* Exact Top-K of every row (operator contract, Section 2.1; phases of Sections 4.2-4.4).
+ *
+ *   scores      packed FP32 rows; base address 16-byte aligned; read-only; NaN-free by
+ *               contract (a NaN pattern is still ranked deterministically by its bits)
+ *   row_starts  [num_rows] element offset of row r in `scores` (any value >= 0; rows need
+ *               not be aligned and must not overlap the end of the allocation)
+ *   row_lengths [num_rows] valid length L_r; a negative length is treated as 0
+ *   K           1 <= K <= HPCTOPK_MAX_K
+ *   out_idx     [num_rows, K] row-major.  For each row the min(K, L_r) ROW-LOCAL indices of
+ *               its largest scores, in unspecified order, followed by -1 sentinels.  Scores
+ *               are ordered by the monotone key of their bit patterns (-0.0 below +0.0,
+ *               +-inf and subnormals numerically); equal scores are taken lowest index
+ *               first, so the index set is unique.
+ *   out_val     [num_rows, K] the selected scores (bit copies) in the same slots, -inf in
+ *               sentinel slots; may be NULL
+ *   workspace   >= hpctopk_workspace_bytes(num_rows, K) bytes, 256-byte aligned; contents
+ *               need not be initialised; calls that may overlap on the device need
+ *               distinct workspaces
+ *   stream      all work is enqueued on `stream` (one small memset and one kernel whose
+ *               launch geometry depends only on num_rows, K and the device); nothing is
+ *               read back, so the call can be captured in a CUDA graph and replayed with
+ *               new contents in the same buffers
+ *
+ * Returns HPCTOPK_OK or an error code; on error nothing was enqueued.  num_rows == 0 is OK. */
+int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
+                   int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                   void* workspace, hpctopk_stream_t stream);
+
+/* Enqueue a copy of the workspace's counters into `host_out` (host memory).  The caller
+ * synchronises `stream` before reading.  Section 4.5 defines the rates these counters
+ * measure (p_band, p_exact). */
+int hpctopk_read_stats(const void* workspace, hpctopk_stats* host_out, hpctopk_stream_t stream);
+
+/* Enqueue a copy of the per-row records of the last call into `host_out`
+ * (host memory, num_rows entries).  The caller synchronises `stream`. */
+int hpctopk_read_row_info(const void* workspace, int32_t num_rows, hpctopk_row_info* host_out,
+                          hpctopk_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HPCTOPK_H_ */

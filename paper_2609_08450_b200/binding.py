@@ -1,0 +1,152 @@
+"""ctypes binding of libhpctopk.so: the same entry points as include/hpctopk.h.
+
+Argument marshalling only.  Every step of the selection runs inside the CUDA
+library; there is no Python or CPU fallback, and a missing library is an error.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhpctopk.so")
+
+HPCTOPK_OK = 0
+HPCTOPK_MAX_K = 4096
+ROUTE_NAMES = ("short", "direct", "primary", "band", "recovery", "overflow")
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("rows_by_route", ctypes.c_uint64 * 6), ("rows_split", ctypes.c_uint64),
+                ("tasks", ctypes.c_uint64), ("candidates_sum", ctypes.c_uint64),
+                ("candidates_max", ctypes.c_uint64), ("elements_sampled", ctypes.c_uint64),
+                ("elements_scanned", ctypes.c_uint64), ("elements_valid", ctypes.c_uint64),
+                ("error_flags", ctypes.c_uint64), ("reserved", ctypes.c_uint64 * 2)]
+
+    def as_dict(self):
+        d = {f"rows_{n}": int(self.rows_by_route[i]) for i, n in enumerate(ROUTE_NAMES)}
+        for name in ("rows_split", "tasks", "candidates_sum", "candidates_max", "elements_sampled",
+                     "elements_scanned", "elements_valid", "error_flags"):
+            d[name] = int(getattr(self, name))
+        return d
+
+
+ROW_INFO_DTYPE = np.dtype([("route", np.int32), ("tau", np.int32), ("c_tau0", np.int32),
+                           ("c_final", np.int32)])
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2609_08450_b200.build` "
+                               "(there is no fallback implementation)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        L.hpctopk_version.restype = ctypes.c_int
+        L.hpctopk_status_string.argtypes = [ctypes.c_int]
+        L.hpctopk_status_string.restype = ctypes.c_char_p
+        L.hpctopk_workspace_bytes.argtypes = [i32, i32]
+        L.hpctopk_workspace_bytes.restype = ctypes.c_size_t
+        L.hpctopk_query_policy.argtypes = [i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.hpctopk_query_policy.restype = ctypes.c_int
+        L.hpctopk_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
+        L.hpctopk_select.restype = ctypes.c_int
+        L.hpctopk_read_stats.argtypes = [vp, ctypes.POINTER(Stats), vp]
+        L.hpctopk_read_stats.restype = ctypes.c_int
+        L.hpctopk_read_row_info.argtypes = [vp, i32, vp, vp]
+        L.hpctopk_read_row_info.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+class HpcTopkError(RuntimeError):
+    def __init__(self, status):
+        self.status = status
+        super().__init__(f"hpctopk status {status}: {hpctopk_status_string(status)}")
+
+
+def hpctopk_version():
+    return int(lib().hpctopk_version())
+
+
+def hpctopk_status_string(status):
+    return lib().hpctopk_status_string(int(status)).decode()
+
+
+def hpctopk_workspace_bytes(max_num_rows, K):
+    return int(lib().hpctopk_workspace_bytes(int(max_num_rows), int(K)))
+
+
+def hpctopk_query_policy(K, L):
+    """(stride, capacity, route) the selector applies at rank K to a row of length L."""
+    s, c, r = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    st = lib().hpctopk_query_policy(int(K), int(L), ctypes.byref(s), ctypes.byref(c), ctypes.byref(r))
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    return s.value, c.value, r.value
+
+
+def hpctopk_select_raw(scores_ptr, row_starts_ptr, row_lengths_ptr, num_rows, K, out_idx_ptr,
+                       out_val_ptr, workspace_ptr, stream_ptr):
+    """The C entry point on raw addresses; returns the status code."""
+    return int(lib().hpctopk_select(scores_ptr, row_starts_ptr, row_lengths_ptr, int(num_rows), int(K),
+                                    out_idx_ptr, out_val_ptr, workspace_ptr, stream_ptr))
+
+
+def hpctopk_select(scores, row_starts, row_lengths, K, out_idx=None, out_val=None, workspace=None,
+                   stream=None, want_values=True):
+    """Select on CUDA tensors.  Allocates outputs / workspace with torch when not given.
+
+    scores fp32 1-D, row_starts / row_lengths int32 [M]; returns (out_idx [M, K] int32,
+    out_val [M, K] fp32 or None, workspace uint8 tensor).
+    """
+    import torch
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.is_contiguous()
+    assert row_starts.dtype == torch.int32 and row_lengths.dtype == torch.int32
+    M = int(row_lengths.numel())
+    dev = scores.device
+    if out_idx is None:
+        out_idx = torch.empty((M, K), dtype=torch.int32, device=dev)
+    if out_val is None and want_values:
+        out_val = torch.empty((M, K), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(max(hpctopk_workspace_bytes(M, K), 256), dtype=torch.uint8, device=dev)
+    if stream is None:
+        stream = torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        st = hpctopk_select_raw(scores.data_ptr(), row_starts.data_ptr(), row_lengths.data_ptr(), M, K,
+                                out_idx.data_ptr(), out_val.data_ptr() if out_val is not None else None,
+                                workspace.data_ptr(), stream.cuda_stream)
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    return out_idx, out_val, workspace
+
+
+def hpctopk_read_stats(workspace, stream=None):
+    """Counters of the last call on `workspace` (synchronises the stream)."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream(workspace.device)
+    out = Stats()
+    st = lib().hpctopk_read_stats(workspace.data_ptr(), ctypes.byref(out), stream.cuda_stream)
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    stream.synchronize()
+    return out.as_dict()
+
+
+def hpctopk_read_row_info(workspace, num_rows, stream=None):
+    """Per-row records of the last call on `workspace` as a structured numpy array."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream(workspace.device)
+    out = np.zeros(num_rows, dtype=ROW_INFO_DTYPE)
+    st = lib().hpctopk_read_row_info(workspace.data_ptr(), int(num_rows), out.ctypes.data, stream.cuda_stream)
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    stream.synchronize()
+    return out

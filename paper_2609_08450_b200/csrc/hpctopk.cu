@@ -1,0 +1,836 @@
+// hpctopk: exact Top-K over ragged FP32 score rows, hand-written for sm_100a.
+//
+// One persistent kernel.  CTAs claim tasks (a whole row, or one contiguous segment of a long
+// row) from a device counter; everything that depends on row lengths is decided on the device,
+// so the launch geometry is a function of (num_rows, K, device) only.
+//
+// Per row (notation of Sections 4.2-4.4 of the paper):
+//   Phase 1  stride-s view -> 2048-bin coarse histogram (11 leading bits of the fp16 key) ->
+//            tau_0, tau_1 -> inclusive FP32 cutoffs (as ordered keys)
+//   Phase 2  one complete-row pass: key <= cutoff ? append (key, index) to shared memory,
+//            count C(tau_0), add to the leading-digit histogram
+//   Phase 3  radix refinement 11+11+10 over the admitted tail, continued over the index bits
+//            when the final equal-key group is larger than the remaining quota
+//   recovery band pass for tau_1; storage-free full-radix select over the whole row otherwise
+//
+// Keys: kd(x) is the descending sortable key (smaller key = larger score), kd = u for a set
+// sign bit and u ^ 0x7FFFFFFF otherwise, u the raw bits.
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/hpctopk.h"
+
+namespace {
+
+constexpr int kBins = 2048;            // B_c and the widest refinement digit
+constexpr int kSplitRowsMax = 512;     // rows beyond this are never split (enough row parallelism)
+constexpr int kSegMinElems = 16384;    // shortest segment worth a CTA
+constexpr int kTasksPerCta = 2;        // split target: tasks >= kTasksPerCta * grid
+
+// workspace layout (bytes)
+constexpr size_t kOffCtrl = 0;                       // uint32 task_counter
+constexpr size_t kOffStats = 256;                    // hpctopk_stats (128 B)
+constexpr size_t kOffSplit = 512;                    // arrive[512], count[512]
+constexpr size_t kZeroBytes = kOffSplit + 2 * kSplitRowsMax * sizeof(uint32_t);
+constexpr size_t kOffRowInfo = 8192;
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline int capacity_for(int K) { return 4 * K > 4096 ? 4 * K : 4096; }
+__host__ __device__ inline int stride_for(int K) {
+  int s = 1;
+  while (s * 2 <= 128 && s * 2 * 16 <= K) s *= 2;
+  return s;
+}
+
+struct Params {
+  const float* scores;
+  const int32_t* row_starts;
+  const int32_t* row_lengths;
+  int32_t num_rows;
+  int32_t K;
+  int32_t* out_idx;
+  float* out_val;
+  unsigned char* ws;
+  int32_t cap;
+  int32_t stride;
+  int32_t q0, q1;
+  int32_t split_enabled;
+};
+
+struct Shared {
+  uint32_t hist[kBins];
+  uint32_t warp_sums[32];
+  uint32_t cand_count;
+  uint32_t out_count;
+  int32_t loc_bin[2];
+  uint32_t loc_below[2];
+  uint32_t loc_at[2];
+  uint32_t cutd[2];
+  int32_t task;
+  uint32_t bcast0;
+  uint32_t bcast1;
+  uint32_t seg_len_vec;     // vectors per segment unit (split table)
+  uint32_t total_tasks;
+};
+
+// Dynamic shared memory: [Shared][ckd: cap u32][cidx: cap u32][seg_base: kSplitRowsMax + 1 u32].
+// Device functions re-derive these pointers from the extern array (instead of receiving
+// generic pointers) so that loads, stores and atomics compile to shared-space instructions.
+extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ Shared& SH() { return *reinterpret_cast<Shared*>(smem_raw); }
+__device__ __forceinline__ uint32_t* CKD() {
+  return reinterpret_cast<uint32_t*>(smem_raw + ((sizeof(Shared) + 15) / 16 * 16));
+}
+
+// ---------------------------------------------------------------- keys and the coarse map
+__device__ __forceinline__ uint32_t kd_of_bits(uint32_t u) {
+  return u ^ (~(uint32_t)((int32_t)u >> 31) & 0x7FFFFFFFu);
+}
+__device__ __forceinline__ uint32_t bits_of_kd(uint32_t kd) {
+  return (kd & 0x80000000u) ? kd : (kd ^ 0x7FFFFFFFu);
+}
+// c(x) of Eq. "coarse-map", evaluated from the descending key.  NaN patterns (outside the
+// contract) are placed by sign so that the map stays monotone in the key.
+__device__ __forceinline__ int coarse_bin_of_kd(uint32_t kd) {
+  const uint32_t u = bits_of_kd(kd);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (u >> 31) ? (kBins - 1) : 0;
+  const uint32_t h = __half_as_ushort(__float2half_rn(__uint_as_float(u)));
+  const uint32_t asc = (h & 0x8000u) ? (h ^ 0xFFFFu) : (h | 0x8000u);
+  return (int)((0xFFFFu - asc) >> 5);
+}
+// Largest descending key whose coarse bin is <= tau: the inclusive FP32 endpoint of the
+// admitted prefix.  Bisection with the same map the histogram used, so the two cannot disagree.
+__device__ __noinline__ uint32_t cutoff_of_bin(int tau) {
+  uint32_t lo = 0u, hi = 0xFFFFFFFFu;     // c(lo) = 0 <= tau always; find max kd with c <= tau
+  while (lo < hi) {
+    const uint32_t mid = lo + (hi - lo) / 2u + 1u;
+    if (coarse_bin_of_kd(mid) <= tau) lo = mid; else hi = mid - 1u;
+  }
+  return lo;
+}
+
+// ---------------------------------------------------------------- block primitives
+template <int THREADS>
+__device__ __forceinline__ uint32_t warp_inclusive_scan(uint32_t v) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, v, d);
+    if (lane >= d) v += n;
+  }
+  return v;
+}
+
+// For up to two quotas: min{b : H(b) >= quota} over the inclusive prefix of sh.hist, with
+// H(b-1) ("below") and h(b) ("at").  loc_bin stays -1 when the histogram total is short.
+// Contains block barriers; every thread must call it.  Leaves sh.hist unchanged.
+template <int THREADS>
+__device__ void locate(Shared& sh, uint32_t quota0, uint32_t quota1, int nq) {
+  constexpr int BPT = kBins / THREADS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t h[BPT];
+  uint32_t sum = 0;
+#pragma unroll
+  for (int b = 0; b < BPT; ++b) { h[b] = sh.hist[tid * BPT + b]; sum += h[b]; }
+  const uint32_t incl = warp_inclusive_scan<THREADS>(sum);
+  if (lane == 31) sh.warp_sums[warp] = incl;
+  if (tid < 2) sh.loc_bin[tid] = -1;
+  __syncthreads();
+  uint32_t woff = 0;
+  for (int w = 0; w < warp; ++w) woff += sh.warp_sums[w];
+  const uint32_t excl = woff + incl - sum;
+  for (int qi = 0; qi < nq; ++qi) {
+    const uint32_t quota = qi ? quota1 : quota0;
+    if (excl < quota && quota <= excl + sum) {
+      uint32_t run = excl;
+#pragma unroll
+      for (int b = 0; b < BPT; ++b) {
+        if (run < quota && run + h[b] >= quota) {
+          sh.loc_bin[qi] = tid * BPT + b; sh.loc_below[qi] = run; sh.loc_at[qi] = h[b];
+        }
+        run += h[b];
+      }
+    }
+  }
+  __syncthreads();
+}
+
+template <int THREADS>
+__device__ __forceinline__ void clear_hist(Shared& sh) {
+  for (int b = threadIdx.x; b < kBins; b += THREADS) sh.hist[b] = 0;
+}
+
+// Warp-aggregated append of admitted elements: one shared-memory reservation per warp.
+// Every lane of the warp must call it.  Entries beyond the capacity are counted, not stored.
+template <bool HIST>
+__device__ __forceinline__ void append_candidate(bool pred, uint32_t kd, uint32_t idx, Shared& sh,
+                                                 uint32_t* ckd, uint32_t* cidx, uint32_t cap) {
+  const uint32_t m = __ballot_sync(0xFFFFFFFFu, pred);
+  if (m) {
+    const int lane = threadIdx.x & 31;
+    const int leader = __ffs(m) - 1;
+    uint32_t base = 0;
+    if (lane == leader) base = atomicAdd(&sh.cand_count, (uint32_t)__popc(m));
+    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (pred) {
+      const uint32_t pos = base + __popc(m & ((1u << lane) - 1u));
+      if (pos < cap) { ckd[pos] = kd; cidx[pos] = idx; }
+      if (HIST) atomicAdd(&sh.hist[kd >> 21], 1u);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- Phase 2: the complete-row pass
+// Scans global elements [e0, e1) of `scores`; row-local index = e - g0.
+//   BAND = false: admit kd <= cut_hi.            (A(tau_0), Eq. "candidate-set")
+//   BAND = true : admit cut_lo < kd <= cut_hi.   (the band of Eq. "rescue-band")
+template <int THREADS, int U, bool BAND>
+__device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
+                           uint32_t cut_lo, uint32_t cut_hi, uint32_t cap) {
+  Shared& sh = SH();
+  uint32_t* const ckd = CKD();
+  uint32_t* const cidx = ckd + cap;
+  const int tid = threadIdx.x;
+  auto admit = [&](uint32_t kd) -> bool {
+    return BAND ? (kd > cut_lo && kd <= cut_hi) : (kd <= cut_hi);
+  };
+  if (e1 <= e0) return;
+  int64_t b0 = (e0 + 3) & ~(int64_t)3;      // first 16-byte aligned element
+  int64_t b1 = e1 & ~(int64_t)3;            // end of the last whole vector
+  if (b0 > b1) { b0 = e1; b1 = e1; }        // range holds no whole vector
+  // ragged edges: at most 3 + 3 scalar elements, handled by warp 0
+  if (tid < 32) {
+    const int64_t head_end = b0 < e1 ? b0 : e1;
+    const int nhead = (int)(head_end - e0);
+    const int ntail = (int)(e1 - (b1 > head_end ? b1 : head_end));
+    int64_t e = -1;
+    if (tid < nhead) e = e0 + tid;
+    else if (tid >= 8 && tid - 8 < ntail) e = e1 - ntail + (tid - 8);
+    uint32_t kd = 0;
+    bool pred = false;
+    if (e >= 0) { kd = kd_of_bits(__float_as_uint(__ldg(scores + e))); pred = admit(kd); }
+    append_candidate<true>(pred, kd, (uint32_t)(e - g0), sh, ckd, cidx, cap);
+  }
+  const int64_t nvec = (b1 - b0) >> 2;
+  if (nvec <= 0) return;
+  const float4* __restrict__ vp = reinterpret_cast<const float4*>(scores + b0);
+  const uint32_t idx0 = (uint32_t)(b0 - g0);
+  constexpr int TILE = THREADS * U;
+  const int64_t nfull = nvec / TILE;
+
+  auto load_tile = [&](float4 (&buf)[U], const float4* p) {
+#pragma unroll
+    for (int j = 0; j < U; ++j) buf[j] = __ldcs(p + j * THREADS);
+  };
+  auto process_tile = [&](const float4 (&buf)[U], uint32_t ibase) {
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const uint32_t i = ibase + (uint32_t)(j * THREADS * 4);
+      const uint32_t k0 = kd_of_bits(__float_as_uint(buf[j].x));
+      const uint32_t k1 = kd_of_bits(__float_as_uint(buf[j].y));
+      const uint32_t k2 = kd_of_bits(__float_as_uint(buf[j].z));
+      const uint32_t k3 = kd_of_bits(__float_as_uint(buf[j].w));
+      append_candidate<true>(admit(k0), k0, i + 0, sh, ckd, cidx, cap);
+      append_candidate<true>(admit(k1), k1, i + 1, sh, ckd, cidx, cap);
+      append_candidate<true>(admit(k2), k2, i + 2, sh, ckd, cidx, cap);
+      append_candidate<true>(admit(k3), k3, i + 3, sh, ckd, cidx, cap);
+    }
+  };
+
+  // Two register tiles: the loads of one are in flight while the other is classified.
+  float4 A[U], B[U];
+  const float4* p = vp + tid;
+  uint32_t ib = idx0 + (uint32_t)(tid << 2);
+  uint32_t left = (uint32_t)nfull;
+  if (left > 0) load_tile(A, p);
+  while (left >= 2) {
+    load_tile(B, p + TILE);
+    process_tile(A, ib);
+    if (left > 2) load_tile(A, p + 2 * TILE);
+    process_tile(B, ib + TILE * 4);
+    p += 2 * TILE;
+    ib += 2 * TILE * 4;
+    left -= 2;
+  }
+  if (left == 1) process_tile(A, ib);
+  // remainder: fewer than TILE vectors, block-uniform trip count
+  for (int64_t vb = nfull * TILE; vb < nvec; vb += THREADS) {
+    const int64_t v = vb + tid;
+    const bool in = v < nvec;
+    float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (in) f = __ldcs(vp + v);
+    const uint32_t i = idx0 + (uint32_t)(v << 2);
+    const uint32_t k0 = kd_of_bits(__float_as_uint(f.x));
+    const uint32_t k1 = kd_of_bits(__float_as_uint(f.y));
+    const uint32_t k2 = kd_of_bits(__float_as_uint(f.z));
+    const uint32_t k3 = kd_of_bits(__float_as_uint(f.w));
+    append_candidate<true>(in && admit(k0), k0, i + 0, sh, ckd, cidx, cap);
+    append_candidate<true>(in && admit(k1), k1, i + 1, sh, ckd, cidx, cap);
+    append_candidate<true>(in && admit(k2), k2, i + 2, sh, ckd, cidx, cap);
+    append_candidate<true>(in && admit(k3), k3, i + 3, sh, ckd, cidx, cap);
+  }
+}
+
+// ---------------------------------------------------------------- element sources for selection
+// A source visits every element once per pass, calling f(valid, kd, idx) with a block-uniform
+// trip count (so f may use warp collectives).
+struct CandidateSource {          // the admitted tail held in shared memory
+  uint32_t cap;
+  uint32_t n;
+  template <int THREADS, typename F>
+  __device__ __forceinline__ void for_each(F f) const {
+    const uint32_t* const ckd = CKD();
+    const uint32_t* const cidx = ckd + cap;
+    for (uint32_t b = 0; b < n; b += THREADS) {
+      const uint32_t i = b + threadIdx.x;
+      const bool v = i < n;
+      f(v, v ? ckd[i] : 0u, v ? cidx[i] : 0u);
+    }
+  }
+};
+
+struct RowSource {                // the complete row in global memory (recovery)
+  const float* scores;
+  int64_t g0, g1;
+  template <int THREADS, typename F>
+  __device__ __forceinline__ void for_each(F f) const {
+    const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
+    for (int64_t base = va; base < vb; base += THREADS) {
+      const int64_t v = base + threadIdx.x;
+      const int64_t e = v << 2;
+      const bool in = v < vb;
+      const bool full = in && e >= g0 && e + 4 <= g1;
+      float x[4] = {0.f, 0.f, 0.f, 0.f};
+      bool ok[4] = {false, false, false, false};
+      if (full) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(scores + e));
+        x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+        ok[0] = ok[1] = ok[2] = ok[3] = true;
+      } else if (in) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          ok[j] = (e + j >= g0) && (e + j < g1);
+          if (ok[j]) x[j] = __ldg(scores + e + j);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) f(ok[j], kd_of_bits(__float_as_uint(x[j])), (uint32_t)(e + j - g0));
+    }
+  }
+};
+
+// ---------------------------------------------------------------- Phase 3 and the output commit
+// Radix selection of the `K` best elements of a source under the composite order
+// (kd ascending, index ascending): digits 11+11+10 of kd (Section 4.4), then, only if the final
+// equal-key group exceeds the remaining quota, 11+11+10 of the index.  Each round is
+// prefix -> boundary digit -> k_{j+1} = k_j - |R_j| (Eqs. "digit-boundary", "refine-recurrence");
+// the frontier Q_j is the set of elements matching the prefix chosen so far.  Selected elements
+// are committed in one final pass: composite >> shift <= prefix.
+// When `hist_ready`, sh.hist already holds the leading-digit histogram of the source.
+template <int THREADS, typename Source>
+__device__ __noinline__ void select_and_emit(const Source src, uint32_t K, bool hist_ready,
+                                             int32_t* out_idx, float* out_val) {
+  Shared& sh = SH();
+  const int shifts[6] = {53, 42, 32, 21, 10, 0};
+  const int widths[6] = {11, 11, 10, 11, 11, 10};
+  uint64_t prefix = 0;
+  int prev_shift = 64;
+  uint32_t k_rem = K;
+#pragma unroll 1
+  for (int j = 0; j < 6; ++j) {
+    const int shift = shifts[j];
+    const uint32_t mask = (1u << widths[j]) - 1u;
+    if (!(j == 0 && hist_ready)) {
+      __syncthreads();
+      clear_hist<THREADS>(sh);
+      __syncthreads();
+      src.template for_each<THREADS>([&](bool valid, uint32_t kd, uint32_t idx) {
+        if (valid) {
+          const uint64_t comp = ((uint64_t)kd << 32) | idx;
+          if (j == 0 || (comp >> prev_shift) == prefix)
+            atomicAdd(&sh.hist[(uint32_t)(comp >> shift) & mask], 1u);
+        }
+      });
+    }
+    __syncthreads();
+    locate<THREADS>(sh, k_rem, 0, 1);
+    const int b = sh.loc_bin[0];
+    const uint32_t below = sh.loc_below[0], at = sh.loc_at[0];
+    if (b < 0) break;                       // cannot happen for a certified state; keeps the loop finite
+    k_rem -= below;
+    prefix = (prefix << widths[j]) | (uint32_t)b;
+    prev_shift = shift;
+    if (at == k_rem) break;                 // the whole boundary group is taken
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) sh.out_count = 0;
+  __syncthreads();
+  src.template for_each<THREADS>([&](bool valid, uint32_t kd, uint32_t idx) {
+    const uint64_t comp = ((uint64_t)kd << 32) | idx;
+    const bool pred = valid && (prev_shift < 64) && ((comp >> prev_shift) <= prefix);
+    const uint32_t m = __ballot_sync(0xFFFFFFFFu, pred);
+    if (m) {
+      const int lane = threadIdx.x & 31;
+      const int leader = __ffs(m) - 1;
+      uint32_t base = 0;
+      if (lane == leader) base = atomicAdd(&sh.out_count, (uint32_t)__popc(m));
+      base = __shfl_sync(0xFFFFFFFFu, base, leader);
+      if (pred) {
+        const uint32_t slot = base + __popc(m & ((1u << lane) - 1u));
+        if (slot < K) {
+          out_idx[slot] = (int32_t)idx;
+          if (out_val) out_val[slot] = __uint_as_float(bits_of_kd(kd));
+        }
+      }
+    }
+  });
+  __syncthreads();
+}
+
+// ---------------------------------------------------------------- per-row bookkeeping
+__device__ __forceinline__ hpctopk_stats* stats_of(unsigned char* ws) {
+  return reinterpret_cast<hpctopk_stats*>(ws + kOffStats);
+}
+__device__ __forceinline__ void add64(uint64_t* p, uint64_t v) {
+  atomicAdd(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
+}
+__device__ __forceinline__ void max64(uint64_t* p, uint64_t v) {
+  atomicMax(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
+}
+__device__ void record_row(const Params& P, int row, int route, int tau, uint32_t c0, uint32_t cfin,
+                           uint64_t scanned, uint64_t sampled, uint64_t L) {
+  if (threadIdx.x != 0) return;
+  hpctopk_stats* st = stats_of(P.ws);
+  add64(&st->rows_by_route[route], 1);
+  if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND) {
+    add64(&st->candidates_sum, cfin);
+    max64(&st->candidates_max, cfin);
+  }
+  if (scanned) add64(&st->elements_scanned, scanned);
+  if (sampled) add64(&st->elements_sampled, sampled);
+  add64(&st->elements_valid, L);
+  int4 info = make_int4(route, tau, (int)c0, (int)cfin);
+  reinterpret_cast<int4*>(P.ws + kOffRowInfo)[row] = info;
+}
+
+// Phase 1 (Section 4.2): sample view -> coarse histogram -> tau_0, tau_1 -> cutoffs in sh.cutd.
+// Returns false when the view cannot support the requested sample ranks.
+template <int THREADS>
+__device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_t L, int& tau_pack) {
+  Shared& sh = SH();
+  const int s = P.stride;
+  const int bits = 31 - __clz(s);
+  const int a = bits ? (int)(__brev((uint32_t)(row & (s - 1))) >> (32 - bits)) : 0;   // pi_s: bit reversal
+  const int64_t n_view = L > a ? (L - a + s - 1) / s : 0;
+  tau_pack = -1;
+  if (n_view < P.q1) return false;
+  __syncthreads();
+  clear_hist<THREADS>(sh);
+  __syncthreads();
+  const float* __restrict__ rowp = P.scores + g0 + a;
+  for (int64_t t = threadIdx.x; t < n_view; t += THREADS) {
+    const uint32_t kd = kd_of_bits(__float_as_uint(__ldg(rowp + t * s)));
+    atomicAdd(&sh.hist[coarse_bin_of_kd(kd)], 1u);
+  }
+  __syncthreads();
+  locate<THREADS>(sh, (uint32_t)P.q0, (uint32_t)P.q1, 2);
+  const int tau0 = sh.loc_bin[0], tau1 = sh.loc_bin[1];
+  if (threadIdx.x == 0) sh.cutd[0] = cutoff_of_bin(tau0);
+  if (threadIdx.x == 32) sh.cutd[1] = cutoff_of_bin(tau1);
+  __syncthreads();
+  tau_pack = tau0 | (tau1 << 16);
+  return true;
+}
+
+template <int THREADS>
+__device__ void emit_short_row(const Params& P, int row, int64_t g0, int64_t L) {
+  int32_t* oi = P.out_idx + (int64_t)row * P.K;
+  float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
+  for (int i = threadIdx.x; i < P.K; i += THREADS) {
+    const bool v = i < L;
+    oi[i] = v ? i : -1;
+    if (ov) ov[i] = v ? __ldg(P.scores + g0 + i) : __uint_as_float(0xFF800000u);
+  }
+}
+
+// Everything after the primary pass of a sampled row: certification branch (Section 4.3),
+// band extension, refinement or exact recovery, output commit.  On entry the shared candidate
+// arrays hold min(C0, cap) entries of A(tau_0) and sh.hist their leading-digit histogram iff
+// `hist_ready`.
+template <int THREADS, int U>
+__device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t L, uint32_t C0,
+                                   bool hist_ready, int tau_pack, uint64_t scanned, uint64_t sampled) {
+  Shared& sh = SH();
+  int32_t* oi = P.out_idx + (int64_t)row * P.K;
+  float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
+  const uint32_t K = (uint32_t)P.K, cap = (uint32_t)P.cap;
+  int route;
+  uint32_t cfin = 0;
+  if (C0 > cap) {
+    route = HPCTOPK_ROUTE_OVERFLOW;
+  } else if (C0 >= K) {
+    route = HPCTOPK_ROUTE_PRIMARY;
+    cfin = C0;
+  } else {
+    // band extension: append tau_0 < c(x) <= tau_1 and extend the histogram (Eq. "rescue-hist")
+    if (!hist_ready) {
+      __syncthreads();
+      clear_hist<THREADS>(sh);
+      __syncthreads();
+      CandidateSource cs{cap, C0};
+      cs.template for_each<THREADS>([&](bool v, uint32_t kd, uint32_t) { if (v) atomicAdd(&sh.hist[kd >> 21], 1u); });
+      hist_ready = true;
+    }
+    __syncthreads();
+    scan_range<THREADS, U, true>(P.scores, g0, g0, g0 + L, sh.cutd[0], sh.cutd[1], cap);
+    __syncthreads();
+    scanned += (uint64_t)L;
+    const uint32_t C1 = sh.cand_count;
+    if (C1 > cap) route = HPCTOPK_ROUTE_OVERFLOW;
+    else if (C1 >= K) { route = HPCTOPK_ROUTE_BAND; cfin = C1; }
+    else route = HPCTOPK_ROUTE_RECOVERY;
+  }
+  if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND) {
+    CandidateSource cs{cap, cfin};
+    select_and_emit<THREADS>(cs, K, hist_ready, oi, ov);
+  } else {
+    RowSource rs{P.scores, g0, g0 + L};
+    select_and_emit<THREADS>(rs, K, false, oi, ov);
+    scanned += 4ull * (uint64_t)L;          // three digit passes and the commit pass, at least
+  }
+  record_row(P, row, route, tau_pack, C0, cfin, scanned, sampled, (uint64_t)L);
+}
+
+// A row owned by one CTA from Phase 1 to the output commit.
+template <int THREADS, int U>
+__device__ void process_row(const Params& P, int row) {
+  Shared& sh = SH();
+  const int64_t g0 = P.row_starts[row];
+  int64_t L = P.row_lengths[row];
+  if (L < 0) L = 0;
+  const uint32_t K = (uint32_t)P.K, cap = (uint32_t)P.cap;
+  int32_t* oi = P.out_idx + (int64_t)row * P.K;
+  float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
+  if (L <= (int64_t)K) {
+    emit_short_row<THREADS>(P, row, g0, L);
+    record_row(P, row, HPCTOPK_ROUTE_SHORT, -1, 0, 0, (uint64_t)L, 0, (uint64_t)L);
+    return;
+  }
+  __syncthreads();
+  if (L <= (int64_t)cap) {
+    // direct route: the whole row is the admitted tail (C = L), refined on chip
+    clear_hist<THREADS>(sh);
+    if (threadIdx.x == 0) sh.cand_count = 0;
+    __syncthreads();
+    scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, 0xFFFFFFFFu, cap);
+    __syncthreads();
+    CandidateSource cs{cap, (uint32_t)L};
+    select_and_emit<THREADS>(cs, K, true, oi, ov);
+    record_row(P, row, HPCTOPK_ROUTE_DIRECT, -1, (uint32_t)L, (uint32_t)L, (uint64_t)L, 0, (uint64_t)L);
+    return;
+  }
+  int tau_pack;
+  if (!phase1<THREADS>(P, row, g0, L, tau_pack)) {
+    RowSource rs{P.scores, g0, g0 + L};
+    select_and_emit<THREADS>(rs, K, false, oi, ov);
+    record_row(P, row, HPCTOPK_ROUTE_RECOVERY, -1, 0, 0, 4ull * (uint64_t)L, 0, (uint64_t)L);
+    return;
+  }
+  const uint64_t sampled = (uint64_t)((L + P.stride - 1) / P.stride);
+  clear_hist<THREADS>(sh);
+  if (threadIdx.x == 0) sh.cand_count = 0;
+  __syncthreads();
+  scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[0], cap);
+  __syncthreads();
+  const uint32_t C0 = sh.cand_count;
+  finish_sampled_row<THREADS, U>(P, row, g0, L, C0, true, tau_pack, (uint64_t)L, sampled);
+}
+
+// One segment of a KV-split row (Section 4.5): same boundary as every other segment of the row,
+// private scan, publication into the row's global candidate range, last arriver finishes.
+template <int THREADS, int U>
+__device__ void process_segment(const Params& P, int row, int seg, int nseg) {
+  Shared& sh = SH();
+  uint32_t* const ckd = CKD();
+  uint32_t* const cidx = ckd + P.cap;
+  const int64_t g0 = P.row_starts[row];
+  const int64_t L = P.row_lengths[row];       // > cap, checked when the table was built
+  const int64_t g1 = g0 + L;
+  const uint32_t cap = (uint32_t)P.cap;
+  uint32_t* arrive = reinterpret_cast<uint32_t*>(P.ws + kOffSplit);
+  uint32_t* rowcnt = arrive + kSplitRowsMax;
+  const size_t cand_off = align_up(kOffRowInfo + (size_t)P.num_rows * sizeof(hpctopk_row_info), 256);
+  uint32_t* gkd = reinterpret_cast<uint32_t*>(P.ws + cand_off) + (size_t)row * 2 * cap;
+  uint32_t* gidx = gkd + cap;
+
+  int tau_pack;
+  const bool usable = phase1<THREADS>(P, row, g0, L, tau_pack);
+  const uint64_t sampled = usable ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
+  // contiguous, 16-byte aligned partition of the row's vectors
+  const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
+  const int64_t per = (vb - va + nseg - 1) / nseg;
+  int64_t e0 = (va + (int64_t)seg * per) << 2, e1 = (va + (int64_t)(seg + 1) * per) << 2;
+  if (e0 < g0) e0 = g0;
+  if (e1 > g1) e1 = g1;
+  if (e1 < e0) e1 = e0;
+  __syncthreads();
+  if (threadIdx.x == 0) sh.cand_count = 0;
+  clear_hist<THREADS>(sh);
+  __syncthreads();
+  if (usable) scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, sh.cutd[0], cap);
+  __syncthreads();
+  const uint32_t Cp = sh.cand_count;
+  if (threadIdx.x == 0) {
+    sh.bcast0 = atomicAdd(&rowcnt[row], Cp);
+    hpctopk_stats* st = stats_of(P.ws);
+    add64(&st->elements_scanned, (uint64_t)(e1 - e0));
+    if (sampled) add64(&st->elements_sampled, sampled);
+  }
+  __syncthreads();
+  const uint32_t base = sh.bcast0;
+  if (base + Cp <= cap) {
+    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) { gkd[base + i] = ckd[i]; gidx[base + i] = cidx[i]; }
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) sh.bcast1 = atomicAdd(&arrive[row], 1u);
+  __syncthreads();
+  if (sh.bcast1 != (uint32_t)(nseg - 1)) return;      // not the last arriver
+  // ---- finisher: C(tau_0) = sum_p C_p, A(tau_0) = union of the published ranges (Eq. "split-reduce")
+  __threadfence();
+  const uint32_t C0 = *reinterpret_cast<volatile uint32_t*>(&rowcnt[row]);
+  if (threadIdx.x == 0) add64(&stats_of(P.ws)->rows_split, 1);
+  if (!usable) {
+    RowSource rs{P.scores, g0, g1};
+    select_and_emit<THREADS>(rs, (uint32_t)P.K, false, P.out_idx + (int64_t)row * P.K,
+                             P.out_val ? P.out_val + (int64_t)row * P.K : nullptr);
+    record_row(P, row, HPCTOPK_ROUTE_RECOVERY, -1, 0, 0, 4ull * (uint64_t)L, 0, (uint64_t)L);
+    return;
+  }
+  if (C0 <= cap) {
+    for (uint32_t i = threadIdx.x; i < C0; i += THREADS) { ckd[i] = __ldcg(gkd + i); cidx[i] = __ldcg(gidx + i); }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) sh.cand_count = C0;
+  __syncthreads();
+  finish_sampled_row<THREADS, U>(P, row, g0, L, C0, false, tau_pack, 0, 0);
+}
+
+// ---------------------------------------------------------------- the persistent kernel
+template <int THREADS, int U, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) {
+  Shared& sh = SH();
+  uint32_t* const seg_base = CKD() + 2 * P.cap;                 // [kSplitRowsMax + 1], only when splitting
+  uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl);
+  const int tid = threadIdx.x;
+
+  uint32_t total_tasks = (uint32_t)P.num_rows;
+  uint32_t seg_unit = 0;
+  if (P.split_enabled) {
+    // Device-side ragged dispatch: every CTA derives the same task table from row_lengths.
+    constexpr int RPT = (kSplitRowsMax + THREADS - 1) / THREADS;
+    unsigned long long mine = 0;
+    for (int j = 0; j < RPT; ++j) {
+      const int r = tid * RPT + j;
+      if (r < P.num_rows) { const int64_t L = P.row_lengths[r]; if (L > P.cap) mine += (unsigned long long)L; }
+    }
+    // block sum of sampled-row elements
+    for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
+    if ((tid & 31) == 0) { sh.hist[2 * (tid >> 5)] = (uint32_t)mine; sh.hist[2 * (tid >> 5) + 1] = (uint32_t)(mine >> 32); }
+    __syncthreads();
+    unsigned long long total = 0;
+    for (int w = 0; w < THREADS / 32; ++w) total += (unsigned long long)sh.hist[2 * w] | ((unsigned long long)sh.hist[2 * w + 1] << 32);
+    const unsigned long long target = (unsigned long long)gridDim.x * kTasksPerCta;
+    unsigned long long S = (total + target - 1) / target;
+    if (S < (unsigned long long)kSegMinElems) S = kSegMinElems;
+    S = (S + 4095ull) / 4096ull * 4096ull;
+    seg_unit = (uint32_t)S;
+    __syncthreads();
+    uint32_t cnt[RPT];
+    uint32_t sum = 0;
+    for (int j = 0; j < RPT; ++j) {
+      const int r = tid * RPT + j;
+      cnt[j] = 0;
+      if (r < P.num_rows) {
+        const int64_t L = P.row_lengths[r];
+        cnt[j] = (L > P.cap) ? (uint32_t)((L + (int64_t)S - 1) / (int64_t)S) : 1u;
+      }
+      sum += cnt[j];
+    }
+    const uint32_t incl = warp_inclusive_scan<THREADS>(sum);
+    if ((tid & 31) == 31) sh.warp_sums[tid >> 5] = incl;
+    __syncthreads();
+    uint32_t woff = 0;
+    for (int w = 0; w < (tid >> 5); ++w) woff += sh.warp_sums[w];
+    uint32_t run = woff + incl - sum;
+    for (int j = 0; j < RPT; ++j) {
+      const int r = tid * RPT + j;
+      if (r < P.num_rows) seg_base[r] = run;
+      run += cnt[j];
+      if (r == P.num_rows - 1) { seg_base[P.num_rows] = run; sh.total_tasks = run; }
+    }
+    __syncthreads();
+    total_tasks = sh.total_tasks;
+  }
+
+  uint32_t task = blockIdx.x;                       // first wave: direct assignment
+  while (task < total_tasks) {
+    if (P.split_enabled) {
+      // largest r with seg_base[r] <= task
+      int lo = 0, hi = P.num_rows - 1;
+      while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (seg_base[mid] <= task) lo = mid; else hi = mid - 1; }
+      const int row = lo;
+      const int nseg = (int)(seg_base[row + 1] - seg_base[row]);
+      if (nseg <= 1) process_row<THREADS, U>(P, row);
+      else process_segment<THREADS, U>(P, row, (int)(task - seg_base[row]), nseg);
+    } else {
+      process_row<THREADS, U>(P, (int)task);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      sh.task = (int32_t)(gridDim.x + atomicAdd(task_counter, 1u));
+      add64(&stats_of(P.ws)->tasks, 1);
+    }
+    __syncthreads();
+    task = (uint32_t)sh.task;
+  }
+  (void)seg_unit;
+}
+
+// ---------------------------------------------------------------- host side
+struct DeviceInfo {
+  bool ready = false;
+  int sm_count = 0;
+  int ctas_per_sm[3] = {0, 0, 0};   // by capacity class
+};
+DeviceInfo g_dev[64];
+
+constexpr int kThreads = 512;
+constexpr int kUnroll = 4;
+constexpr int kMinBlocks = 2;
+using KernelFn = void (*)(const Params);
+KernelFn main_kernel() { return hpctopk_kernel<kThreads, kUnroll, kMinBlocks>; }
+
+size_t smem_bytes_for(int cap, bool split) {
+  size_t b = align_up(sizeof(Shared), 16) + (size_t)cap * 8;
+  if (split) b += (kSplitRowsMax + 1) * sizeof(uint32_t);
+  return align_up(b, 16);
+}
+
+int cap_class(int cap) { return cap <= 4096 ? 0 : (cap <= 8192 ? 1 : 2); }
+
+}  // namespace
+
+extern "C" {
+
+int hpctopk_version(void) { return 1000 * 0 + 1; }
+
+const char* hpctopk_status_string(int status) {
+  switch (status) {
+    case HPCTOPK_OK: return "ok";
+    case HPCTOPK_ERR_INVALID_ARG: return "invalid argument";
+    case HPCTOPK_ERR_UNSUPPORTED_K: return "K exceeds HPCTOPK_MAX_K";
+    case HPCTOPK_ERR_MISALIGNED: return "misaligned scores or workspace pointer";
+    case HPCTOPK_ERR_WORKSPACE: return "workspace error";
+    case HPCTOPK_ERR_CUDA: return "CUDA runtime error";
+    case HPCTOPK_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
+  if (max_num_rows < 0 || K < 1 || K > HPCTOPK_MAX_K) return 0;
+  const size_t cap = (size_t)capacity_for(K);
+  const size_t split_rows = max_num_rows < kSplitRowsMax ? (size_t)max_num_rows : (size_t)kSplitRowsMax;
+  size_t b = align_up(kOffRowInfo + (size_t)max_num_rows * sizeof(hpctopk_row_info), 256);
+  b += split_rows * cap * 8;
+  return align_up(b, 256);
+}
+
+int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route) {
+  if (K < 1) return HPCTOPK_ERR_INVALID_ARG;
+  if (K > HPCTOPK_MAX_K) return HPCTOPK_ERR_UNSUPPORTED_K;
+  if (stride) *stride = stride_for(K);
+  if (capacity) *capacity = capacity_for(K);
+  if (route) *route = L <= K ? HPCTOPK_ROUTE_SHORT : (L <= capacity_for(K) ? HPCTOPK_ROUTE_DIRECT : HPCTOPK_ROUTE_PRIMARY);
+  return HPCTOPK_OK;
+}
+
+int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
+                   int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                   void* workspace, hpctopk_stream_t stream) {
+  if (num_rows < 0 || K < 1) return HPCTOPK_ERR_INVALID_ARG;
+  if (K > HPCTOPK_MAX_K) return HPCTOPK_ERR_UNSUPPORTED_K;
+  if (num_rows == 0) return HPCTOPK_OK;
+  if (!scores || !row_starts || !row_lengths || !out_idx || !workspace) return HPCTOPK_ERR_INVALID_ARG;
+  if (((uintptr_t)scores & 15u) || ((uintptr_t)workspace & 255u)) return HPCTOPK_ERR_MISALIGNED;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HPCTOPK_ERR_CUDA;
+  DeviceInfo& di = g_dev[dev];
+  const int cap = capacity_for(K);
+  const bool split = num_rows <= kSplitRowsMax;
+  if (!di.ready) {
+    if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
+    const size_t max_smem = smem_bytes_for(capacity_for(HPCTOPK_MAX_K), true);
+    if (cudaFuncSetAttribute(main_kernel(), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    const int caps[3] = {4096, 8192, capacity_for(HPCTOPK_MAX_K)};
+    for (int c = 0; c < 3; ++c) {
+      int n = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, main_kernel(), kThreads, smem_bytes_for(caps[c], true)) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        return HPCTOPK_ERR_CUDA;
+      }
+      di.ctas_per_sm[c] = n;
+    }
+    di.ready = true;
+  }
+  Params P;
+  P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
+  P.num_rows = num_rows; P.K = K; P.out_idx = out_idx; P.out_val = out_val;
+  P.ws = static_cast<unsigned char*>(workspace);
+  P.cap = cap; P.stride = stride_for(K);
+  P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);      // ceil(1.5 K / s)
+  P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);      // ceil(1.75 K / s)
+  P.split_enabled = split ? 1 : 0;
+  // smem is sized by capacity class so that occupancy (and the grid) depends on K only
+  const int cls = cap_class(cap);
+  const int cls_cap = cls == 0 ? 4096 : (cls == 1 ? 8192 : capacity_for(HPCTOPK_MAX_K));
+  const size_t smem = smem_bytes_for(cls_cap, true);
+  const int grid = di.sm_count * di.ctas_per_sm[cls];
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
+  main_kernel()<<<grid, kThreads, smem, st>>>(P);
+  if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
+  return HPCTOPK_OK;
+}
+
+int hpctopk_read_stats(const void* workspace, hpctopk_stats* host_out, hpctopk_stream_t stream) {
+  if (!workspace || !host_out) return HPCTOPK_ERR_INVALID_ARG;
+  if (cudaMemcpyAsync(host_out, static_cast<const unsigned char*>(workspace) + kOffStats, sizeof(hpctopk_stats),
+                      cudaMemcpyDeviceToHost, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return HPCTOPK_ERR_CUDA;
+  }
+  return HPCTOPK_OK;
+}
+
+int hpctopk_read_row_info(const void* workspace, int32_t num_rows, hpctopk_row_info* host_out,
+                          hpctopk_stream_t stream) {
+  if (!workspace || !host_out || num_rows < 0) return HPCTOPK_ERR_INVALID_ARG;
+  if (num_rows == 0) return HPCTOPK_OK;
+  if (cudaMemcpyAsync(host_out, static_cast<const unsigned char*>(workspace) + kOffRowInfo,
+                      (size_t)num_rows * sizeof(hpctopk_row_info), cudaMemcpyDeviceToHost,
+                      reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return HPCTOPK_ERR_CUDA;
+  }
+  return HPCTOPK_OK;
+}
+
+}  // extern "C"

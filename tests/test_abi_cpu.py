@@ -1,0 +1,68 @@
+"""Host-side checks that need no GPU: the library loads, exports every declared symbol,
+and its host-only entry points and argument validation behave as the header says."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from oracle import sampled_steps as S
+from paper_2609_08450_b200 import binding as B, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return B.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "hpctopk.h")).read()
+    names = set(re.findall(r"\b(hpctopk_[a-z_]+)\s*\(", header))
+    assert {"hpctopk_select", "hpctopk_workspace_bytes", "hpctopk_read_stats", "hpctopk_read_row_info",
+            "hpctopk_query_policy", "hpctopk_status_string", "hpctopk_version"} <= names
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_host_only_entry_points(lib):
+    assert B.hpctopk_version() >= 1
+    assert B.hpctopk_status_string(0) == "ok"
+    assert "K" in B.hpctopk_status_string(2)
+    assert B.hpctopk_workspace_bytes(-1, 2048) == 0
+    assert B.hpctopk_workspace_bytes(8, 0) == 0
+    assert B.hpctopk_workspace_bytes(8, B.HPCTOPK_MAX_K + 1) == 0
+    small, big = B.hpctopk_workspace_bytes(8, 2048), B.hpctopk_workspace_bytes(1 << 20, 2048)
+    assert small % 256 == 0 and 0 < small < big
+    # bounded: a constant plus 16 bytes per row, whatever the row width
+    assert big - B.hpctopk_workspace_bytes(512, 2048) <= 16 * (1 << 20) + 4096
+
+
+def test_policy_mirror_matches_the_reading_of_the_paper(lib):
+    for K in (1, 8, 31, 32, 512, 1000, 1024, 2048, 4096):
+        s, cap, _ = B.hpctopk_query_policy(K, 10 ** 6)
+        assert s == S.stride_for(K) and cap == S.capacity_for(K)
+        assert B.hpctopk_query_policy(K, K)[2] == S.ROUTE_SHORT
+        assert B.hpctopk_query_policy(K, K + 1)[2] == S.ROUTE_DIRECT
+        assert B.hpctopk_query_policy(K, cap)[2] == S.ROUTE_DIRECT
+        assert B.hpctopk_query_policy(K, cap + 1)[2] == S.ROUTE_PRIMARY
+    assert B.hpctopk_query_policy(2048, 1)[0] == 128
+    with pytest.raises(B.HpcTopkError):
+        B.hpctopk_query_policy(0, 5)
+
+
+def test_argument_validation_returns_before_any_cuda_call(lib):
+    f = B.hpctopk_select_raw
+    ok_ptr = 0x1000
+    assert f(ok_ptr, ok_ptr, ok_ptr, 0, 8, ok_ptr, None, ok_ptr, None) == 0          # no rows: nothing to do
+    assert f(ok_ptr, ok_ptr, ok_ptr, -1, 8, ok_ptr, None, ok_ptr, None) == 1
+    assert f(ok_ptr, ok_ptr, ok_ptr, 4, 0, ok_ptr, None, ok_ptr, None) == 1
+    assert f(ok_ptr, ok_ptr, ok_ptr, 4, B.HPCTOPK_MAX_K + 1, ok_ptr, None, ok_ptr, None) == 2
+    assert f(None, ok_ptr, ok_ptr, 4, 8, ok_ptr, None, ok_ptr, None) == 1
+    assert f(ok_ptr, ok_ptr, ok_ptr, 4, 8, None, None, ok_ptr, None) == 1
+    assert f(ok_ptr + 4, ok_ptr, ok_ptr, 4, 8, ok_ptr, None, ok_ptr, None) == 3      # scores not 16 B aligned
+    assert f(ok_ptr, ok_ptr, ok_ptr, 4, 8, ok_ptr, None, ok_ptr + 16, None) == 3     # workspace not 256 B aligned
+    st = B.Stats()
+    assert lib.hpctopk_read_stats(None, ctypes.byref(st), None) == 1

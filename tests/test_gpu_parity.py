@@ -1,0 +1,176 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, bit-exact,
+on the five workload recipes and on edge cases."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sampled_steps as S
+from paper_2609_08450_b200 import binding as B, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _common():
+    from tests import gpu_common
+    return gpu_common
+
+
+def _batch_from_rows(rows, name="custom"):
+    lengths = np.array([len(r) for r in rows], dtype=np.int64)
+    flat = np.concatenate([np.asarray(r, dtype=np.float32) for r in rows]) if len(rows) else np.zeros(0, np.float32)
+    if flat.size == 0:
+        flat = np.zeros(4, np.float32)      # keep a valid device pointer; no row reads it
+    starts = np.zeros(len(rows), dtype=np.int64)
+    starts[1:] = np.cumsum(lengths[:-1])
+    return W.Batch(name, torch.from_numpy(flat).to(DEV), torch.from_numpy(starts.astype(np.int32)).to(DEV),
+                   torch.from_numpy(lengths.astype(np.int32)).to(DEV))
+
+
+def test_config1_small_ragged():
+    stats, info, _, _ = _common().check_batch(W.config1(DEV), 2048, check_trace=True)
+    assert stats["rows_short"] >= 2
+
+
+def test_tiny_rows_every_length_and_rank():
+    rng = np.random.default_rng(1)
+    alphabet = np.array([-np.inf, -0.0, 0.0, 1.0, np.inf, -2.5, 3.25], dtype=np.float32)
+    rows = [alphabet[rng.integers(0, len(alphabet), size=L)] for L in range(0, 71) for _ in range(3)]
+    batch = _batch_from_rows(rows)
+    for K in range(1, 9):
+        _common().check_batch(batch, K)
+    _common().check_batch(batch, 64)
+
+
+def test_config2_decode_batch():
+    stats, info, _, _ = _common().check_batch(W.config2(DEV), 2048, check_trace=True)
+    assert stats["rows_split"] > 0                      # 64 rows < SM count: the KV-split mapping runs
+    assert stats["rows_primary"] + stats["rows_band"] >= 56
+
+
+def test_config3_prefill_chunk_full_size_sampled_rows():
+    batch = W.config3(DEV)
+    assert batch.num_rows == 4096 and batch.total_elements == 528484352
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([[0, 1, 2, 4095, 4094], rng.integers(0, 4096, size=91)]))
+    stats, info, got_idx, _ = _common().check_batch(batch, 2048, rows=rows, check_trace=False)
+    # properties that hold for every row at any size
+    lengths = batch.row_lengths.cpu().numpy()
+    assert (got_idx >= 0).all() and (got_idx < lengths[:, None]).all()
+    srt = np.sort(got_idx, axis=1)
+    assert (np.diff(srt, axis=1) > 0).all()             # K distinct indices per row
+    assert stats["rows_split"] == 0
+    assert stats["rows_primary"] + stats["rows_band"] + stats["rows_recovery"] + stats["rows_overflow"] == 4096
+
+
+@pytest.mark.parametrize("K", [2048, 4096])
+def test_config4_long_context(K):
+    stats, info, _, _ = _common().check_batch(W.config4(DEV), K, check_trace=True)
+    assert stats["rows_split"] == 16
+
+
+@pytest.mark.parametrize("K", [512, 1024, 2048])
+def test_config5_adversarial(K):
+    stride, _, _ = B.hpctopk_query_policy(K, 65536)
+    stats, info, _, _ = _common().check_batch(W.config5(K, stride, DEV), K, check_trace=True)
+    assert stats["rows_recovery"] + stats["rows_overflow"] > 0
+
+
+@pytest.mark.parametrize("K", [512, 2048])
+def test_adversarial_long_rows_split_and_single(K):
+    """The structured kinds at lengths that reach the sampled path, once with few rows
+    (KV-split) and once with more rows than the split limit (one CTA per row)."""
+    stride, cap, _ = B.hpctopk_query_policy(K, 10 ** 6)
+    rng = np.random.default_rng(K)
+    rows = []
+    for kind in W.ADVERSARIAL_KINDS:
+        for L in (cap + 1, 4 * K + 3, 50001, 200000):
+            rows.append(W.adversarial_row(kind, L, K, stride, rng))
+    _common().check_batch(_batch_from_rows(rows, "adv_long_few"), K, check_trace=True)
+    many = [W.adversarial_row(W.ADVERSARIAL_KINDS[i % 8], int(rng.integers(cap + 1, 30000)), K, stride, rng)
+            for i in range(560)]
+    stats, _, _, _ = _common().check_batch(_batch_from_rows(many, "adv_long_many"), K, check_trace=True)
+    assert stats["rows_split"] == 0
+
+
+def test_many_rows_without_values_and_determinism():
+    batch = W.config1(DEV, seed=77, num_rows=700, max_len=40000, K=1024)
+    c = _common()
+    stats, _, idx1, _ = c.check_batch(batch, 1024, want_values=False)
+    _, _, idx2, _ = c.check_batch(batch, 1024, want_values=False)
+    assert np.array_equal(np.sort(idx1, axis=1), np.sort(idx2, axis=1))
+
+
+def test_forced_underfill_reaches_band_and_recovery():
+    """Rows built so that the sampled residue class misses part of the upper tail."""
+    K = 2048
+    stride, cap, _ = B.hpctopk_query_policy(K, 10 ** 6)
+    rng = np.random.default_rng(5)
+    rows = []
+    for r in range(64):
+        L = 100000 + r
+        x = rng.normal(size=L).astype(np.float32)
+        a = S.phase_offset(r, stride)
+        # lift a set of positions the view never sees, so the sample under-estimates the tail
+        hide = np.arange(L)
+        hide = hide[(hide % stride) != a][: 3000 + 40 * r]
+        x[hide] += np.float32(50.0)
+        rows.append(x)
+    many = rows * 9                      # > split limit: single-CTA path
+    c = _common()
+    s1, _, _, _ = c.check_batch(_batch_from_rows(rows, "underfill_few"), K, check_trace=True)
+    s2, _, _, _ = c.check_batch(_batch_from_rows(many, "underfill_many"), K, check_trace=True)
+    for s in (s1, s2):
+        assert s["rows_band"] + s["rows_recovery"] + s["rows_overflow"] > 0
+
+
+def test_nan_patterns_are_ranked_by_their_bits():
+    x = np.random.default_rng(2).normal(size=30000).astype(np.float32)
+    x[[5, 77, 20000]] = np.nan
+    x[[9, 10]] = np.array([0xFFC00000, 0xFF800001], dtype=np.uint32).view(np.float32)
+    _common().check_batch(_batch_from_rows([x, x[:3000], x[:100]]), 2048)
+
+
+def test_negative_and_zero_lengths_are_empty_rows():
+    rows = [np.arange(10, dtype=np.float32), np.arange(5000, dtype=np.float32)]
+    batch = _batch_from_rows(rows)
+    batch.row_lengths = torch.tensor([-3, 5000, 0], dtype=torch.int32, device=DEV)
+    batch.row_starts = torch.tensor([0, 10, 0], dtype=torch.int32, device=DEV)
+    _common().check_batch(batch, 16)
+
+
+def test_cuda_graph_replay_with_new_lengths_in_the_same_buffers():
+    K = 2048
+    a = W.config1(DEV, seed=11, num_rows=24, max_len=90000)
+    b = W.config1(DEV, seed=12, num_rows=24, max_len=90000)
+    n = max(a.scores.numel(), b.scores.numel())
+    scores = torch.zeros(n, device=DEV)
+    starts = torch.zeros(24, dtype=torch.int32, device=DEV)
+    lengths = torch.zeros(24, dtype=torch.int32, device=DEV)
+    out_idx = torch.empty((24, K), dtype=torch.int32, device=DEV)
+    out_val = torch.empty((24, K), dtype=torch.float32, device=DEV)
+    ws = torch.empty(B.hpctopk_workspace_bytes(24, K), dtype=torch.uint8, device=DEV)
+
+    def load(batch):
+        scores[: batch.scores.numel()].copy_(batch.scores)
+        starts.copy_(batch.row_starts)
+        lengths.copy_(batch.row_lengths)
+
+    load(a)
+    B.hpctopk_select(scores, starts, lengths, K, out_idx, out_val, ws)       # first call outside capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=side):
+        B.hpctopk_select(scores, starts, lengths, K, out_idx, out_val, ws, stream=torch.cuda.current_stream())
+    from oracle import native
+    from tests.helpers import assert_rows_match
+    for batch in (a, b, a):
+        load(batch)
+        out_idx.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        s, st, ln = batch.host()
+        want, _, _ = native.topk_stable_sort(s, st, ln, K)
+        assert_rows_match(s, st, ln, K, out_idx.cpu().numpy(), out_val.cpu().numpy(), want)
