@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of the exact ragged Top-K selector (one JSON line on rank 0).
+
+A "step" is one hpctopk_select call over one batch of synthetic score rows: the whole
+hot path (sample, fused complete-row pass, refinement, recovery routes, output commit).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config3|config2|config4]
+  python bench.py --impl reference ...      # the CPU oracle, timed on a bounded sample
+
+Default workload: config 3 of the benchmark spec (prefill chunk, 4096 causal rows of
+126977..131072 scores, K = 2048; 2.11 GB of FP32 scores, larger than L2).  With N > 1
+(torchrun, one rank per GPU) every rank selects its own batch of the same recipe
+(weak scaling, no data-path collective); timings are CUDA-event sums, max over ranks.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+K = 2048
+# DRAM bytes per score element of the dominant kernel, from the ncu capture summarised in
+# profiles/hpctopk_kernel_config3_small.md (dram__bytes_read.sum + dram__bytes_write.sum over
+# the valid elements of the captured launch; traffic grows in proportion to the elements).
+NCU_DRAM_BYTES_PER_ELEMENT = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._thread = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
+                parts = [p.strip() for p in out.stdout.strip().split(",")]
+                if len(parts) >= 6:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+def make_batch(workload, device, rank):
+    from paper_2609_08450_b200 import workloads as W
+    seed_shift = 1000 * rank
+    if workload == "config3":
+        return W.config3(device, seed=W.BASE_SEED + 3 + seed_shift)
+    if workload == "config2":
+        return W.config2(device, seed=W.BASE_SEED + 2 + seed_shift)
+    if workload == "config4":
+        return W.config4(device, seed=W.BASE_SEED + 4 + seed_shift)
+    raise ValueError(workload)
+
+
+WORKLOAD_TEXT = {
+    "config3": "BASELINE.json configs[2]: prefill chunk, 4096 causal rows L=126977..131072, K=2048",
+    "config2": "BASELINE.json configs[1]: decode batch, 64 rows L~U[16384,131072], K=2048",
+    "config4": "BASELINE.json configs[3]: long context, 16 rows L~U[524288,1048576], K=2048",
+}
+
+
+def oracle_sample_rows(num_rows, sample_rows):
+    """Evenly spaced row sample for the CPU oracle."""
+    n = min(sample_rows, num_rows)
+    return np.unique(np.linspace(0, num_rows - 1, n).astype(np.int64))
+
+
+def time_oracle(scores, starts, lengths, rows):
+    from oracle import native
+    t0 = time.perf_counter()
+    _, _, used = native.topk_stable_sort(scores, starts[rows], lengths[rows], K)
+    dt = time.perf_counter() - t0
+    return dt, int(np.clip(lengths[rows], 0, None).sum()), used
+
+
+def run_reference(args, rank, world):
+    """The CPU oracle as it stands, on the host cores, on a bounded sample per step."""
+    if rank != 0:
+        return
+    from oracle import native
+    from paper_2609_08450_b200 import workloads as W
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    if dev == "cuda":
+        batch = make_batch(args.workload, dev, 0)
+    else:   # no GPU: a reduced copy of the same recipe keeps the arm runnable
+        batch = W.config3("cpu", num_rows=64, seq_len=16384, offset=16384 - 65, heads=8, dim=32, slab=8)
+    scores, starts, lengths = batch.host()
+    rows = oracle_sample_rows(len(lengths), args.ref_rows)
+    for _ in range(args.warmup):
+        time_oracle(scores, starts, lengths, rows[: max(1, len(rows) // 8)])
+    total_t, total_e, used = 0.0, 0, 1
+    for _ in range(args.steps):
+        dt, ne, used = time_oracle(scores, starts, lengths, rows)
+        total_t += dt
+        total_e += ne
+    value = total_e / total_t
+    sample = f"{len(rows)} evenly spaced rows of the workload per step ({total_e // args.steps} score elements)"
+    line = {"impl": "reference", "metric": "score elements/s, exact Top-K K=2048", "value": value,
+            "unit": "score elements/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "rows_per_s": len(rows) * args.steps / total_t,
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "K": K, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "score elements/s", "cores": used, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "score elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config3", choices=list(WORKLOAD_TEXT))
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-rows", type=int, default=192, help="rows per step of the CPU oracle arm")
+    ap.add_argument("--cpu-baseline-rows", type=int, default=1024)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch.distributed as dist
+    from paper_2609_08450_b200 import binding as B, build, sharding
+    if not os.path.exists(B.LIB_PATH):
+        build.build()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    batch = make_batch(args.workload, dev, rank)
+    M, n_elem = batch.num_rows, batch.total_elements
+    out_idx = torch.empty((M, K), dtype=torch.int32, device=dev)
+    out_val = torch.empty((M, K), dtype=torch.float32, device=dev)
+    ws = torch.empty(B.hpctopk_workspace_bytes(M, K), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    input_bytes = 4 * n_elem
+    flush = None
+    if input_bytes < 512 * 1024 * 1024:            # smaller than a few L2s: flush between steps
+        flush = torch.empty(512 * 1024 * 1024 // 4, dtype=torch.float32, device=dev)
+
+    def step():
+        B.hpctopk_select(batch.scores, batch.row_starts, batch.row_lengths, K, out_idx, out_val, ws, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        if flush is not None:
+            flush.fill_(1.0)
+        step()
+    barrier()
+    starts_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        for i in range(args.steps):
+            if flush is not None:
+                flush.fill_(1.0)
+            starts_ev[i].record(stream)
+            step()
+            ends_ev[i].record(stream)
+        barrier()
+    ms = [s.elapsed_time(e) for s, e in zip(starts_ev, ends_ev)]
+    total_ms = sharding.max_over_ranks(sum(ms), dev)
+    all_elems = sharding.sum_over_ranks(n_elem, dev)
+    all_rows = sharding.sum_over_ranks(M, dev)
+    stats = B.hpctopk_read_stats(ws, stream)
+
+    # end to end: host buffers in, host buffers out, copies inside the timed region
+    h_scores = batch.scores.cpu().pin_memory()
+    h_starts = batch.row_starts.cpu().pin_memory()
+    h_lengths = batch.row_lengths.cpu().pin_memory()
+    h_idx = torch.empty((M, K), dtype=torch.int32).pin_memory()
+    h_val = torch.empty((M, K), dtype=torch.float32).pin_memory()
+    d_scores = torch.empty_like(batch.scores)
+    d_starts = torch.empty_like(batch.row_starts)
+    d_lengths = torch.empty_like(batch.row_lengths)
+
+    def e2e_step():
+        d_scores.copy_(h_scores, non_blocking=True)
+        d_starts.copy_(h_starts, non_blocking=True)
+        d_lengths.copy_(h_lengths, non_blocking=True)
+        B.hpctopk_select(d_scores, d_starts, d_lengths, K, out_idx, out_val, ws, stream)
+        h_idx.copy_(out_idx, non_blocking=True)
+        h_val.copy_(out_val, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
+    h2d = 4 * n_elem + 8 * M
+    d2h = 8 * M * K
+
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        value = all_elems * args.steps / (total_ms * 1e-3)
+        local_ms = float(np.mean(ms))
+        achieved = 4.0 * n_elem / (local_ms * 1e-3) / 1e9        # GB/s of algorithmic score bytes
+        traffic = None if NCU_DRAM_BYTES_PER_ELEMENT is None else NCU_DRAM_BYTES_PER_ELEMENT * n_elem
+        line = {
+            "metric": "score elements/s, exact Top-K K=2048", "value": value, "unit": "score elements/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "rows_per_s": all_rows * args.steps / (total_ms * 1e-3),
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "K": K, "rows_per_gpu": M,
+                       "score_elements_per_gpu": n_elem,
+                       "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps (512 MB write)"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                         "frac_of_nominal_8TBs": achieved / 8000.0,
+                         "algorithmic_bytes": "4 bytes per valid score (one complete-row read)"},
+            "e2e": {"value": all_elems * args.e2e_steps / (e2e_ms * 1e-3), "unit": "score elements/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": args.steps,
+            "clocks": clocks.summary(),
+            "routes": {k: v for k, v in stats.items() if k.startswith("rows_")},
+            "row_equivalent_reads": (stats["elements_scanned"] + stats["elements_sampled"]) / max(stats["elements_valid"], 1),
+        }
+        if not args.no_cpu_baseline and world == 1:
+            scores, starts, lengths = h_scores.numpy(), h_starts.numpy(), h_lengths.numpy()
+            rows = oracle_sample_rows(M, args.cpu_baseline_rows)
+            dt, ne, used = time_oracle(scores, starts, lengths, rows)
+            line["cpu_baseline"] = {"value": ne / dt, "unit": "score elements/s", "cores": used, "kind": "oracle",
+                                    "sample": f"{len(rows)} evenly spaced rows of the workload ({ne} score elements), "
+                                              f"std::stable_sort per row, OpenMP over rows"}
+        else:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

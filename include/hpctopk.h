@@ -57,6 +57,11 @@ typedef struct {
   uint64_t elements_scanned;  /* score reads issued by complete-row passes (all routes) */
   uint64_t elements_valid;    /* sum of valid row lengths */
   uint64_t error_flags;       /* nonzero: an internal invariant was violated */
+  uint64_t cycles_phase1;     /* SM clock cycles summed over CTAs: Phase 1 (sample to cutoffs) */
+  uint64_t cycles_scan;       /* ... the primary complete-row pass (Phase 2) */
+  uint64_t cycles_finish;     /* ... certification branch, band/recovery, Phase 3, output commit */
+  uint64_t cycles_total;      /* ... whole tasks, from claim to completion */
+  uint64_t cycles_detail[8];  /* finer split of the above, for tuning runs (meaning may change) */
   uint64_t reserved[2];
 } hpctopk_stats;
 

@@ -9,7 +9,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libhpctopk.so")
+LIB_PATH = os.environ.get("HPCTOPK_LIB", os.path.join(_HERE, "libhpctopk.so"))
 
 HPCTOPK_OK = 0
 HPCTOPK_MAX_K = 4096
@@ -21,13 +21,18 @@ class Stats(ctypes.Structure):
                 ("tasks", ctypes.c_uint64), ("candidates_sum", ctypes.c_uint64),
                 ("candidates_max", ctypes.c_uint64), ("elements_sampled", ctypes.c_uint64),
                 ("elements_scanned", ctypes.c_uint64), ("elements_valid", ctypes.c_uint64),
-                ("error_flags", ctypes.c_uint64), ("reserved", ctypes.c_uint64 * 2)]
+                ("error_flags", ctypes.c_uint64), ("cycles_phase1", ctypes.c_uint64),
+                ("cycles_scan", ctypes.c_uint64), ("cycles_finish", ctypes.c_uint64),
+                ("cycles_total", ctypes.c_uint64), ("cycles_detail", ctypes.c_uint64 * 8),
+                ("reserved", ctypes.c_uint64 * 2)]
 
     def as_dict(self):
         d = {f"rows_{n}": int(self.rows_by_route[i]) for i, n in enumerate(ROUTE_NAMES)}
         for name in ("rows_split", "tasks", "candidates_sum", "candidates_max", "elements_sampled",
-                     "elements_scanned", "elements_valid", "error_flags"):
+                     "elements_scanned", "elements_valid", "error_flags", "cycles_phase1", "cycles_scan",
+                     "cycles_finish", "cycles_total"):
             d[name] = int(getattr(self, name))
+        d["cycles_detail"] = [int(v) for v in self.cycles_detail]
         return d
 
 

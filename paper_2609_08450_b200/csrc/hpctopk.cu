@@ -19,8 +19,13 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <stdlib.h>
 
 #include "../../include/hpctopk.h"
+
+#ifndef HPCTOPK_EXPERIMENT
+#define HPCTOPK_EXPERIMENT 0
+#endif
 
 namespace {
 
@@ -31,13 +36,19 @@ constexpr int kTasksPerCta = 2;        // split target: tasks >= kTasksPerCta * 
 
 // workspace layout (bytes)
 constexpr size_t kOffCtrl = 0;                       // uint32 task_counter
-constexpr size_t kOffStats = 256;                    // hpctopk_stats (128 B)
+constexpr size_t kOffStats = 256;                    // hpctopk_stats (176 B)
 constexpr size_t kOffSplit = 512;                    // arrive[512], count[512]
 constexpr size_t kZeroBytes = kOffSplit + 2 * kSplitRowsMax * sizeof(uint32_t);
 constexpr size_t kOffRowInfo = 8192;
+constexpr int kPrefetchAheadBytes = 65536;   // L2 prefetch distance inside a row's scan
+constexpr int kPrefetchHeadBytes = 131072;   // bytes of the next task's range warmed in L2 ahead of time
+constexpr int kMaxGrid = 1024;         // upper bound on resident CTAs (sizes the spill region)
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// Candidate capacity: `capacity_for` entries in total, the first `smem_capacity_for` of them in
+// shared memory and the rest in the CTA's global overflow slice (Section 5.3).
 __host__ __device__ inline int capacity_for(int K) { return 4 * K > 4096 ? 4 * K : 4096; }
+__host__ __device__ inline int smem_capacity_for(int K) { return 2 * K > 2048 ? 2 * K : 2048; }
 __host__ __device__ inline int stride_for(int K) {
   int s = 1;
   while (s * 2 <= 128 && s * 2 * 16 <= K) s *= 2;
@@ -53,7 +64,8 @@ struct Params {
   int32_t* out_idx;
   float* out_val;
   unsigned char* ws;
-  int32_t cap;
+  int32_t cap;          // total candidate capacity (entries)
+  int32_t cap_s;        // entries held in shared memory; the rest spill to the CTA's global slice
   int32_t stride;
   int32_t q0, q1;
   int32_t split_enabled;
@@ -69,19 +81,20 @@ struct Shared {
   uint32_t loc_at[2];
   uint32_t cutd[2];
   int32_t task;
+  int32_t claim;
   uint32_t bcast0;
   uint32_t bcast1;
   uint32_t seg_len_vec;     // vectors per segment unit (split table)
   uint32_t total_tasks;
 };
 
-// Dynamic shared memory: [Shared][ckd: cap u32][cidx: cap u32][seg_base: kSplitRowsMax + 1 u32].
+// Dynamic shared memory: [Shared][cand: cap x (kd, idx) pairs][seg_base: kSplitRowsMax + 1 u32].
 // Device functions re-derive these pointers from the extern array (instead of receiving
 // generic pointers) so that loads, stores and atomics compile to shared-space instructions.
 extern __shared__ __align__(16) unsigned char smem_raw[];
 __device__ __forceinline__ Shared& SH() { return *reinterpret_cast<Shared*>(smem_raw); }
-__device__ __forceinline__ uint32_t* CKD() {
-  return reinterpret_cast<uint32_t*>(smem_raw + ((sizeof(Shared) + 15) / 16 * 16));
+__device__ __forceinline__ uint2* CAND() {
+  return reinterpret_cast<uint2*>(smem_raw + ((sizeof(Shared) + 15) / 16 * 16));
 }
 
 // ---------------------------------------------------------------- keys and the coarse map
@@ -101,12 +114,19 @@ __device__ __forceinline__ int coarse_bin_of_kd(uint32_t kd) {
   return (int)((0xFFFFu - asc) >> 5);
 }
 // Largest descending key whose coarse bin is <= tau: the inclusive FP32 endpoint of the
-// admitted prefix.  Bisection with the same map the histogram used, so the two cannot disagree.
+// admitted prefix.  Searched with the same map the histogram used, so the two cannot disagree.
+// One warp, 32 probes per step (c is non-decreasing in kd, so the probes that pass form a
+// prefix); every lane of the calling warp must take part and receives the result.
 __device__ __noinline__ uint32_t cutoff_of_bin(int tau) {
-  uint32_t lo = 0u, hi = 0xFFFFFFFFu;     // c(lo) = 0 <= tau always; find max kd with c <= tau
-  while (lo < hi) {
-    const uint32_t mid = lo + (hi - lo) / 2u + 1u;
-    if (coarse_bin_of_kd(mid) <= tau) lo = mid; else hi = mid - 1u;
+  const uint32_t lane = threadIdx.x & 31;
+  uint32_t lo = 0u;                         // invariant: c(lo) <= tau  (c(0) = 0)
+#pragma unroll 1
+  for (int b = 27; b >= -3; b -= 5) {
+    const int sh = b < 0 ? 0 : b;
+    const uint32_t nprobe = b < 0 ? 3u : 31u;            // last step resolves the two low bits
+    const uint64_t probe = (uint64_t)lo + ((uint64_t)(lane + 1) << sh);
+    const bool ok = lane < nprobe && probe <= 0xFFFFFFFFull && coarse_bin_of_kd((uint32_t)probe) <= tau;
+    lo += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, ok)) << sh;
   }
   return lo;
 }
@@ -162,56 +182,91 @@ __device__ __forceinline__ void clear_hist(Shared& sh) {
   for (int b = threadIdx.x; b < kBins; b += THREADS) sh.hist[b] = 0;
 }
 
-// Warp-aggregated append of admitted elements: one shared-memory reservation per warp.
-// Every lane of the warp must call it.  Entries beyond the capacity are counted, not stored.
-template <bool HIST>
-__device__ __forceinline__ void append_candidate(bool pred, uint32_t kd, uint32_t idx, Shared& sh,
-                                                 uint32_t* ckd, uint32_t* cidx, uint32_t cap) {
-  const uint32_t m = __ballot_sync(0xFFFFFFFFu, pred);
-  if (m) {
-    const int lane = threadIdx.x & 31;
-    const int leader = __ffs(m) - 1;
-    uint32_t base = 0;
-    if (lane == leader) base = atomicAdd(&sh.cand_count, (uint32_t)__popc(m));
-    base = __shfl_sync(0xFFFFFFFFu, base, leader);
-    if (pred) {
-      const uint32_t pos = base + __popc(m & ((1u << lane) - 1u));
-      if (pos < cap) { ckd[pos] = kd; cidx[pos] = idx; }
-      if (HIST) atomicAdd(&sh.hist[kd >> 21], 1u);
-    }
+// Admission test on raw bits, one integer compare per score (Section 5.3 compares the FP32
+// score with the cutoff directly).  With cu the bit pattern of the cutoff score:
+//   cu >= 0 as int32 (cutoff positive):  admitted  <=>  (int32)u >= (int32)cu
+//   cu <  0          (cutoff negative):  admitted  <=>  u <= cu   (unsigned)
+// Both are (int32)(u ^ flip) >= bound with flip = 0 / 0x7FFFFFFF and bound = cu ^ flip, and
+// both agree with kd(u) <= kd(cu), including signed zeros, infinities and NaN patterns.
+struct Admit {
+  uint32_t flip;
+  int32_t bound;
+  __device__ __forceinline__ explicit Admit(uint32_t cut_kd) {
+    const uint32_t cu = bits_of_kd(cut_kd);
+    flip = (cu & 0x80000000u) ? 0x7FFFFFFFu : 0u;
+    bound = (int32_t)(cu ^ flip);
   }
+  __device__ __forceinline__ bool operator()(uint32_t u) const { return (int32_t)(u ^ flip) >= bound; }
+};
+
+// Where admitted scores go: shared memory first, then this CTA's global overflow slice.
+struct CandCtx {
+  uint32_t cap_s, cap;
+  uint2* spill;
+};
+__device__ __forceinline__ CandCtx cand_ctx(const Params& P) {
+  const size_t cand_off = align_up(kOffRowInfo + (size_t)P.num_rows * sizeof(hpctopk_row_info), 256);
+  const size_t split_rows = P.num_rows < kSplitRowsMax ? P.num_rows : kSplitRowsMax;
+  const size_t spill_off = cand_off + split_rows * (size_t)P.cap * 8;
+  CandCtx c;
+  c.cap_s = (uint32_t)P.cap_s;
+  c.cap = (uint32_t)P.cap;
+  c.spill = reinterpret_cast<uint2*>(P.ws + spill_off) + (size_t)blockIdx.x * (size_t)(P.cap - P.cap_s);
+  return c;
+}
+__device__ __forceinline__ uint2 cand_load(const CandCtx& c, uint32_t i) {
+  return i < c.cap_s ? CAND()[i] : __ldcg(c.spill + (i - c.cap_s));
+}
+__device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v) {
+  if (i < c.cap_s) CAND()[i] = v; else c.spill[i - c.cap_s] = v;
+}
+
+// Append one admitted score: reserve a slot, store (kd, idx), add to the leading-digit histogram
+// (Eq. "first-exact-hist").  Entries beyond the capacity are counted, not stored.
+__device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const CandCtx& c) {
+  Shared& sh = SH();
+  const uint32_t kd = kd_of_bits(u);
+#if HPCTOPK_EXPERIMENT == 2
+  const uint32_t pos = idx & 2047u; sh.cand_count = 3000;
+#else
+  const uint32_t pos = atomicAdd(&sh.cand_count, 1u);
+#endif
+  if (pos < c.cap_s) CAND()[pos] = make_uint2(kd, idx);
+  else if (pos < c.cap) c.spill[pos - c.cap_s] = make_uint2(kd, idx);
+#if HPCTOPK_EXPERIMENT == 0
+  atomicAdd(&sh.hist[kd >> 21], 1u);
+#endif
 }
 
 // ---------------------------------------------------------------- Phase 2: the complete-row pass
 // Scans global elements [e0, e1) of `scores`; row-local index = e - g0.
 //   BAND = false: admit kd <= cut_hi.            (A(tau_0), Eq. "candidate-set")
 //   BAND = true : admit cut_lo < kd <= cut_hi.   (the band of Eq. "rescue-band")
+// Admitted scores are rare (about 1.5 K / L of the row), so the loop spends one compare and one
+// branch per score and leaves everything else to the taken branch.
 template <int THREADS, int U, bool BAND>
 __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
-                           uint32_t cut_lo, uint32_t cut_hi, uint32_t cap) {
-  Shared& sh = SH();
-  uint32_t* const ckd = CKD();
-  uint32_t* const cidx = ckd + cap;
+                                        uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
   const int tid = threadIdx.x;
-  auto admit = [&](uint32_t kd) -> bool {
-    return BAND ? (kd > cut_lo && kd <= cut_hi) : (kd <= cut_hi);
-  };
   if (e1 <= e0) return;
-  int64_t b0 = (e0 + 3) & ~(int64_t)3;      // first 16-byte aligned element
-  int64_t b1 = e1 & ~(int64_t)3;            // end of the last whole vector
-  if (b0 > b1) { b0 = e1; b1 = e1; }        // range holds no whole vector
-  // ragged edges: at most 3 + 3 scalar elements, handled by warp 0
-  if (tid < 32) {
+  const Admit in_hi(cut_hi);
+  const Admit in_lo(cut_lo);                 // BAND: scores admitted by tau_0 are already held
+  auto admit = [&](uint32_t u) -> bool { return BAND ? (in_hi(u) && !in_lo(u)) : in_hi(u); };
+  int64_t b0 = (e0 + 3) & ~(int64_t)3;       // first 16-byte aligned element
+  int64_t b1 = e1 & ~(int64_t)3;             // end of the last whole vector
+  if (b0 > b1) { b0 = e1; b1 = e1; }         // range holds no whole vector
+  // ragged edges: at most 3 + 3 scalar elements
+  if (tid < 16) {
     const int64_t head_end = b0 < e1 ? b0 : e1;
     const int nhead = (int)(head_end - e0);
     const int ntail = (int)(e1 - (b1 > head_end ? b1 : head_end));
     int64_t e = -1;
     if (tid < nhead) e = e0 + tid;
     else if (tid >= 8 && tid - 8 < ntail) e = e1 - ntail + (tid - 8);
-    uint32_t kd = 0;
-    bool pred = false;
-    if (e >= 0) { kd = kd_of_bits(__float_as_uint(__ldg(scores + e))); pred = admit(kd); }
-    append_candidate<true>(pred, kd, (uint32_t)(e - g0), sh, ckd, cidx, cap);
+    if (e >= 0) {
+      const uint32_t u = __float_as_uint(__ldg(scores + e));
+      if (admit(u)) append_candidate(u, (uint32_t)(e - g0), cc);
+    }
   }
   const int64_t nvec = (b1 - b0) >> 2;
   if (nvec <= 0) return;
@@ -220,23 +275,31 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
   constexpr int TILE = THREADS * U;
   const int64_t nfull = nvec / TILE;
 
+  auto classify = [&](const float4& f, uint32_t i) {
+    const uint32_t u0 = __float_as_uint(f.x), u1 = __float_as_uint(f.y);
+    const uint32_t u2 = __float_as_uint(f.z), u3 = __float_as_uint(f.w);
+    if (admit(u0)) append_candidate(u0, i + 0, cc);
+    if (admit(u1)) append_candidate(u1, i + 1, cc);
+    if (admit(u2)) append_candidate(u2, i + 2, cc);
+    if (admit(u3)) append_candidate(u3, i + 3, cc);
+  };
+  // The loads are fed from L2: each thread asks for the lines kPrefetchAheadBytes further on,
+  // so DRAM latency is covered by requests that hold no registers.
+  constexpr int PF_VEC = kPrefetchAheadBytes / 16;
+  const float4* const pf_end = vp + nvec;
   auto load_tile = [&](float4 (&buf)[U], const float4* p) {
 #pragma unroll
-    for (int j = 0; j < U; ++j) buf[j] = __ldcs(p + j * THREADS);
+    for (int j = 0; j < U; ++j) {
+      buf[j] = __ldcs(p + j * THREADS);
+      if (!BAND) {
+        const float4* q = p + j * THREADS + PF_VEC;
+        if (q < pf_end) asm volatile("prefetch.global.L2 [%0];" ::"l"(q));
+      }
+    }
   };
   auto process_tile = [&](const float4 (&buf)[U], uint32_t ibase) {
 #pragma unroll
-    for (int j = 0; j < U; ++j) {
-      const uint32_t i = ibase + (uint32_t)(j * THREADS * 4);
-      const uint32_t k0 = kd_of_bits(__float_as_uint(buf[j].x));
-      const uint32_t k1 = kd_of_bits(__float_as_uint(buf[j].y));
-      const uint32_t k2 = kd_of_bits(__float_as_uint(buf[j].z));
-      const uint32_t k3 = kd_of_bits(__float_as_uint(buf[j].w));
-      append_candidate<true>(admit(k0), k0, i + 0, sh, ckd, cidx, cap);
-      append_candidate<true>(admit(k1), k1, i + 1, sh, ckd, cidx, cap);
-      append_candidate<true>(admit(k2), k2, i + 2, sh, ckd, cidx, cap);
-      append_candidate<true>(admit(k3), k3, i + 3, sh, ckd, cidx, cap);
-    }
+    for (int j = 0; j < U; ++j) classify(buf[j], ibase + (uint32_t)(j * THREADS * 4));
   };
 
   // Two register tiles: the loads of one are in flight while the other is classified.
@@ -255,38 +318,24 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
     left -= 2;
   }
   if (left == 1) process_tile(A, ib);
-  // remainder: fewer than TILE vectors, block-uniform trip count
-  for (int64_t vb = nfull * TILE; vb < nvec; vb += THREADS) {
-    const int64_t v = vb + tid;
-    const bool in = v < nvec;
-    float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (in) f = __ldcs(vp + v);
-    const uint32_t i = idx0 + (uint32_t)(v << 2);
-    const uint32_t k0 = kd_of_bits(__float_as_uint(f.x));
-    const uint32_t k1 = kd_of_bits(__float_as_uint(f.y));
-    const uint32_t k2 = kd_of_bits(__float_as_uint(f.z));
-    const uint32_t k3 = kd_of_bits(__float_as_uint(f.w));
-    append_candidate<true>(in && admit(k0), k0, i + 0, sh, ckd, cidx, cap);
-    append_candidate<true>(in && admit(k1), k1, i + 1, sh, ckd, cidx, cap);
-    append_candidate<true>(in && admit(k2), k2, i + 2, sh, ckd, cidx, cap);
-    append_candidate<true>(in && admit(k3), k3, i + 3, sh, ckd, cidx, cap);
-  }
+  // remainder: fewer than TILE vectors
+  for (int64_t v = nfull * TILE + tid; v < nvec; v += THREADS)
+    classify(__ldcs(vp + v), idx0 + (uint32_t)(v << 2));
 }
 
 // ---------------------------------------------------------------- element sources for selection
 // A source visits every element once per pass, calling f(valid, kd, idx) with a block-uniform
 // trip count (so f may use warp collectives).
-struct CandidateSource {          // the admitted tail held in shared memory
-  uint32_t cap;
+struct CandidateSource {          // the admitted tail: shared memory, then the overflow slice
+  CandCtx cc;
   uint32_t n;
   template <int THREADS, typename F>
   __device__ __forceinline__ void for_each(F f) const {
-    const uint32_t* const ckd = CKD();
-    const uint32_t* const cidx = ckd + cap;
     for (uint32_t b = 0; b < n; b += THREADS) {
       const uint32_t i = b + threadIdx.x;
       const bool v = i < n;
-      f(v, v ? ckd[i] : 0u, v ? cidx[i] : 0u);
+      const uint2 c = v ? cand_load(cc, i) : make_uint2(0u, 0u);
+      f(v, c.x, c.y);
     }
   }
 };
@@ -393,6 +442,9 @@ __device__ __noinline__ void select_and_emit(const Source src, uint32_t K, bool 
 __device__ __forceinline__ hpctopk_stats* stats_of(unsigned char* ws) {
   return reinterpret_cast<hpctopk_stats*>(ws + kOffStats);
 }
+#define TSTAMP(P, k, t_prev) do { if (threadIdx.x == 0) { const long long t_now = clock64(); add64(&stats_of((P).ws)->cycles_detail[k], (uint64_t)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+__device__ __forceinline__ void add64(uint64_t* p, uint64_t v);
+__device__ __forceinline__ hpctopk_stats* stats_of(unsigned char* ws);
 __device__ __forceinline__ void add64(uint64_t* p, uint64_t v) {
   atomicAdd(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
 }
@@ -437,8 +489,13 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   __syncthreads();
   locate<THREADS>(sh, (uint32_t)P.q0, (uint32_t)P.q1, 2);
   const int tau0 = sh.loc_bin[0], tau1 = sh.loc_bin[1];
-  if (threadIdx.x == 0) sh.cutd[0] = cutoff_of_bin(tau0);
-  if (threadIdx.x == 32) sh.cutd[1] = cutoff_of_bin(tau1);
+  if (threadIdx.x < 32) {
+    const uint32_t c0 = cutoff_of_bin(tau0);
+    if (threadIdx.x == 0) sh.cutd[0] = c0;
+  } else if (threadIdx.x < 64) {
+    const uint32_t c1 = cutoff_of_bin(tau1);
+    if (threadIdx.x == 32) sh.cutd[1] = c1;
+  }
   __syncthreads();
   tau_pack = tau0 | (tau1 << 16);
   return true;
@@ -463,6 +520,7 @@ template <int THREADS, int U>
 __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t L, uint32_t C0,
                                    bool hist_ready, int tau_pack, uint64_t scanned, uint64_t sampled) {
   Shared& sh = SH();
+  const CandCtx cc = cand_ctx(P);
   int32_t* oi = P.out_idx + (int64_t)row * P.K;
   float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
   const uint32_t K = (uint32_t)P.K, cap = (uint32_t)P.cap;
@@ -479,12 +537,12 @@ __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t
       __syncthreads();
       clear_hist<THREADS>(sh);
       __syncthreads();
-      CandidateSource cs{cap, C0};
+      CandidateSource cs{cc, C0};
       cs.template for_each<THREADS>([&](bool v, uint32_t kd, uint32_t) { if (v) atomicAdd(&sh.hist[kd >> 21], 1u); });
       hist_ready = true;
     }
     __syncthreads();
-    scan_range<THREADS, U, true>(P.scores, g0, g0, g0 + L, sh.cutd[0], sh.cutd[1], cap);
+    scan_range<THREADS, U, true>(P.scores, g0, g0, g0 + L, sh.cutd[0], sh.cutd[1], cc);
     __syncthreads();
     scanned += (uint64_t)L;
     const uint32_t C1 = sh.cand_count;
@@ -493,7 +551,7 @@ __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t
     else route = HPCTOPK_ROUTE_RECOVERY;
   }
   if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND) {
-    CandidateSource cs{cap, cfin};
+    CandidateSource cs{cc, cfin};
     select_and_emit<THREADS>(cs, K, hist_ready, oi, ov);
   } else {
     RowSource rs{P.scores, g0, g0 + L};
@@ -507,6 +565,7 @@ __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t
 template <int THREADS, int U>
 __device__ void process_row(const Params& P, int row) {
   Shared& sh = SH();
+  const CandCtx cc = cand_ctx(P);
   const int64_t g0 = P.row_starts[row];
   int64_t L = P.row_lengths[row];
   if (L < 0) L = 0;
@@ -524,28 +583,37 @@ __device__ void process_row(const Params& P, int row) {
     clear_hist<THREADS>(sh);
     if (threadIdx.x == 0) sh.cand_count = 0;
     __syncthreads();
-    scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, 0xFFFFFFFFu, cap);
+    scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, 0xFFFFFFFFu, cc);
     __syncthreads();
-    CandidateSource cs{cap, (uint32_t)L};
+    CandidateSource cs{cc, (uint32_t)L};
     select_and_emit<THREADS>(cs, K, true, oi, ov);
     record_row(P, row, HPCTOPK_ROUTE_DIRECT, -1, (uint32_t)L, (uint32_t)L, (uint64_t)L, 0, (uint64_t)L);
     return;
   }
   int tau_pack;
+  const long long t0 = clock64();
   if (!phase1<THREADS>(P, row, g0, L, tau_pack)) {
     RowSource rs{P.scores, g0, g0 + L};
     select_and_emit<THREADS>(rs, K, false, oi, ov);
     record_row(P, row, HPCTOPK_ROUTE_RECOVERY, -1, 0, 0, 4ull * (uint64_t)L, 0, (uint64_t)L);
     return;
   }
+  const long long t1 = clock64();
   const uint64_t sampled = (uint64_t)((L + P.stride - 1) / P.stride);
   clear_hist<THREADS>(sh);
   if (threadIdx.x == 0) sh.cand_count = 0;
   __syncthreads();
-  scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[0], cap);
+  scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[0], cc);
   __syncthreads();
+  const long long t2 = clock64();
   const uint32_t C0 = sh.cand_count;
   finish_sampled_row<THREADS, U>(P, row, g0, L, C0, true, tau_pack, (uint64_t)L, sampled);
+  if (threadIdx.x == 0) {
+    hpctopk_stats* st = stats_of(P.ws);
+    add64(&st->cycles_phase1, (uint64_t)(t1 - t0));
+    add64(&st->cycles_scan, (uint64_t)(t2 - t1));
+    add64(&st->cycles_finish, (uint64_t)(clock64() - t2));
+  }
 }
 
 // One segment of a KV-split row (Section 4.5): same boundary as every other segment of the row,
@@ -553,8 +621,7 @@ __device__ void process_row(const Params& P, int row) {
 template <int THREADS, int U>
 __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   Shared& sh = SH();
-  uint32_t* const ckd = CKD();
-  uint32_t* const cidx = ckd + P.cap;
+  const CandCtx cc = cand_ctx(P);
   const int64_t g0 = P.row_starts[row];
   const int64_t L = P.row_lengths[row];       // > cap, checked when the table was built
   const int64_t g1 = g0 + L;
@@ -562,11 +629,12 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   uint32_t* arrive = reinterpret_cast<uint32_t*>(P.ws + kOffSplit);
   uint32_t* rowcnt = arrive + kSplitRowsMax;
   const size_t cand_off = align_up(kOffRowInfo + (size_t)P.num_rows * sizeof(hpctopk_row_info), 256);
-  uint32_t* gkd = reinterpret_cast<uint32_t*>(P.ws + cand_off) + (size_t)row * 2 * cap;
-  uint32_t* gidx = gkd + cap;
+  uint2* gcand = reinterpret_cast<uint2*>(P.ws + cand_off) + (size_t)row * cap;
 
   int tau_pack;
+  const long long t0 = clock64();
   const bool usable = phase1<THREADS>(P, row, g0, L, tau_pack);
+  const long long t1 = clock64();
   const uint64_t sampled = usable ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
   // contiguous, 16-byte aligned partition of the row's vectors
   const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
@@ -579,19 +647,22 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   if (threadIdx.x == 0) sh.cand_count = 0;
   clear_hist<THREADS>(sh);
   __syncthreads();
-  if (usable) scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, sh.cutd[0], cap);
+  if (usable) scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, sh.cutd[0], cc);
   __syncthreads();
   const uint32_t Cp = sh.cand_count;
+  const long long t2 = clock64();
   if (threadIdx.x == 0) {
     sh.bcast0 = atomicAdd(&rowcnt[row], Cp);
     hpctopk_stats* st = stats_of(P.ws);
+    add64(&st->cycles_phase1, (uint64_t)(t1 - t0));
+    add64(&st->cycles_scan, (uint64_t)(t2 - t1));
     add64(&st->elements_scanned, (uint64_t)(e1 - e0));
     if (sampled) add64(&st->elements_sampled, sampled);
   }
   __syncthreads();
   const uint32_t base = sh.bcast0;
   if (base + Cp <= cap) {
-    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) { gkd[base + i] = ckd[i]; gidx[base + i] = cidx[i]; }
+    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gcand[base + i] = cand_load(cc, i);
   }
   __threadfence();
   __syncthreads();
@@ -610,24 +681,50 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
     return;
   }
   if (C0 <= cap) {
-    for (uint32_t i = threadIdx.x; i < C0; i += THREADS) { ckd[i] = __ldcg(gkd + i); cidx[i] = __ldcg(gidx + i); }
+    for (uint32_t i = threadIdx.x; i < C0; i += THREADS) cand_store(cc, i, __ldcg(gcand + i));
   }
   __syncthreads();
   if (threadIdx.x == 0) sh.cand_count = C0;
   __syncthreads();
   finish_sampled_row<THREADS, U>(P, row, g0, L, C0, false, tau_pack, 0, 0);
+  if (threadIdx.x == 0) add64(&stats_of(P.ws)->cycles_finish, (uint64_t)(clock64() - t2));
 }
 
 // ---------------------------------------------------------------- the persistent kernel
+// Warm the L2 with the stride-s view of a row this CTA will own next, so that its Phase 1 does
+// not start with a DRAM round trip.
+template <int THREADS>
+__device__ __forceinline__ void prefetch_view(const Params& P, int row) {
+  const int64_t g0 = P.row_starts[row];
+  const int64_t L = P.row_lengths[row];
+  if (L <= P.cap) return;
+  const int s = P.stride;
+  const int bits = 31 - __clz(s);
+  const int a = bits ? (int)(__brev((uint32_t)(row & (s - 1))) >> (32 - bits)) : 0;
+  const int64_t n_view = (L - a + s - 1) / s;
+  const float* rowp = P.scores + g0 + a;
+  for (int64_t t = threadIdx.x; t < n_view; t += THREADS)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp + t * s));
+}
+
+// Warm the L2 with the first kPrefetchHeadBytes of the element range [e0, e1) a later task scans.
+template <int THREADS>
+__device__ __forceinline__ void prefetch_head(const Params& P, int64_t e0, int64_t e1) {
+  const char* base = reinterpret_cast<const char*>(P.scores + e0);
+  int64_t bytes = (e1 - e0) * 4;
+  if (bytes > kPrefetchHeadBytes) bytes = kPrefetchHeadBytes;
+  for (int64_t off = (int64_t)threadIdx.x * 128; off < bytes; off += (int64_t)THREADS * 128)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+}
+
 template <int THREADS, int U, int MINB>
 __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) {
   Shared& sh = SH();
-  uint32_t* const seg_base = CKD() + 2 * P.cap;                 // [kSplitRowsMax + 1], only when splitting
+  uint32_t* const seg_base = reinterpret_cast<uint32_t*>(CAND() + P.cap_s);   // [kSplitRowsMax + 1], only when splitting
   uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl);
   const int tid = threadIdx.x;
 
   uint32_t total_tasks = (uint32_t)P.num_rows;
-  uint32_t seg_unit = 0;
   if (P.split_enabled) {
     // Device-side ragged dispatch: every CTA derives the same task table from row_lengths.
     constexpr int RPT = (kSplitRowsMax + THREADS - 1) / THREADS;
@@ -636,7 +733,6 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
       const int r = tid * RPT + j;
       if (r < P.num_rows) { const int64_t L = P.row_lengths[r]; if (L > P.cap) mine += (unsigned long long)L; }
     }
-    // block sum of sampled-row elements
     for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
     if ((tid & 31) == 0) { sh.hist[2 * (tid >> 5)] = (uint32_t)mine; sh.hist[2 * (tid >> 5) + 1] = (uint32_t)(mine >> 32); }
     __syncthreads();
@@ -646,7 +742,6 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
     unsigned long long S = (total + target - 1) / target;
     if (S < (unsigned long long)kSegMinElems) S = kSegMinElems;
     S = (S + 4095ull) / 4096ull * 4096ull;
-    seg_unit = (uint32_t)S;
     __syncthreads();
     uint32_t cnt[RPT];
     uint32_t sum = 0;
@@ -675,8 +770,19 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
     total_tasks = sh.total_tasks;
   }
 
-  uint32_t task = blockIdx.x;                       // first wave: direct assignment
+  // Two statically assigned waves, then completion-order claiming from the device counter.
+  // The claim for the task after next is issued at the top of each task, so its latency and the
+  // L2 warm-up of the next row's view overlap the current row.
+  uint32_t task = blockIdx.x;
+  uint32_t next = blockIdx.x + gridDim.x;
   while (task < total_tasks) {
+    const long long task_t0 = clock64();
+    if (tid == 0) sh.claim = (int32_t)(2u * gridDim.x + atomicAdd(task_counter, 1u));
+    if (!P.split_enabled && next < total_tasks) {
+      prefetch_view<THREADS>(P, (int)next);
+      const int64_t ng0 = P.row_starts[next], nL = P.row_lengths[next];
+      if (nL > P.K) prefetch_head<THREADS>(P, ng0, ng0 + nL);
+    }
     if (P.split_enabled) {
       // largest r with seg_base[r] <= task
       int lo = 0, hi = P.num_rows - 1;
@@ -689,37 +795,50 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
       process_row<THREADS, U>(P, (int)task);
     }
     __syncthreads();
+    const uint32_t claimed = (uint32_t)sh.claim;
     if (tid == 0) {
-      sh.task = (int32_t)(gridDim.x + atomicAdd(task_counter, 1u));
       add64(&stats_of(P.ws)->tasks, 1);
+      add64(&stats_of(P.ws)->cycles_total, (uint64_t)(clock64() - task_t0));
     }
     __syncthreads();
-    task = (uint32_t)sh.task;
+    task = next;
+    next = claimed;
   }
-  (void)seg_unit;
 }
 
 // ---------------------------------------------------------------- host side
+using KernelFn = void (*)(const Params);
+struct Variant {
+  KernelFn fn;
+  int threads;
+};
+// Launch shapes (threads per CTA, register tiles per thread, minimum CTAs per SM).  Index 0 is
+// the default; the others exist for tuning runs (environment variable HPCTOPK_VARIANT).
+const Variant kVariants[] = {
+    {hpctopk_kernel<512, 2, 2>, 512},
+    {hpctopk_kernel<256, 2, 4>, 256},
+    {hpctopk_kernel<256, 4, 3>, 256},
+    {hpctopk_kernel<128, 4, 6>, 128},
+};
+constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
+
 struct DeviceInfo {
   bool ready = false;
   int sm_count = 0;
-  int ctas_per_sm[3] = {0, 0, 0};   // by capacity class
+  int variant = 0;
+  int ctas_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // [split][capacity class]
 };
 DeviceInfo g_dev[64];
 
-constexpr int kThreads = 512;
-constexpr int kUnroll = 4;
-constexpr int kMinBlocks = 2;
-using KernelFn = void (*)(const Params);
-KernelFn main_kernel() { return hpctopk_kernel<kThreads, kUnroll, kMinBlocks>; }
-
-size_t smem_bytes_for(int cap, bool split) {
-  size_t b = align_up(sizeof(Shared), 16) + (size_t)cap * 8;
+size_t smem_bytes_for(int cap_s, bool split) {
+  size_t b = align_up(sizeof(Shared), 16) + (size_t)cap_s * 8;
   if (split) b += (kSplitRowsMax + 1) * sizeof(uint32_t);
   return align_up(b, 16);
 }
 
-int cap_class(int cap) { return cap <= 4096 ? 0 : (cap <= 8192 ? 1 : 2); }
+// Shared memory is sized by capacity class so that occupancy (and the grid) depends on K only.
+int cap_class(int K) { return K <= 1024 ? 0 : (K <= 2048 ? 1 : 2); }
+int class_cap_s(int cls) { return smem_capacity_for(cls == 0 ? 1024 : (cls == 1 ? 2048 : HPCTOPK_MAX_K)); }
 
 }  // namespace
 
@@ -743,9 +862,12 @@ const char* hpctopk_status_string(int status) {
 size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
   if (max_num_rows < 0 || K < 1 || K > HPCTOPK_MAX_K) return 0;
   const size_t cap = (size_t)capacity_for(K);
+  const int cap_s_cls = class_cap_s(cap_class(K));
+  const size_t cap_s = (size_t)cap_s_cls < cap ? (size_t)cap_s_cls : cap;
   const size_t split_rows = max_num_rows < kSplitRowsMax ? (size_t)max_num_rows : (size_t)kSplitRowsMax;
   size_t b = align_up(kOffRowInfo + (size_t)max_num_rows * sizeof(hpctopk_row_info), 256);
-  b += split_rows * cap * 8;
+  b += split_rows * cap * 8;                       // published candidate ranges of split rows
+  b += (size_t)kMaxGrid * (cap - cap_s) * 8;       // one overflow slice per resident CTA
   return align_up(b, 256);
 }
 
@@ -770,42 +892,47 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HPCTOPK_ERR_CUDA;
   DeviceInfo& di = g_dev[dev];
-  const int cap = capacity_for(K);
   const bool split = num_rows <= kSplitRowsMax;
   if (!di.ready) {
     if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
-    const size_t max_smem = smem_bytes_for(capacity_for(HPCTOPK_MAX_K), true);
-    if (cudaFuncSetAttribute(main_kernel(), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
+    const char* env = getenv("HPCTOPK_VARIANT");
+    di.variant = env ? atoi(env) : 0;
+    if (di.variant < 0 || di.variant >= kNumVariants) di.variant = 0;
+    const Variant& v = kVariants[di.variant];
+    const size_t max_smem = smem_bytes_for(class_cap_s(2), true);
+    if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
       cudaGetLastError();
       return HPCTOPK_ERR_CUDA;
     }
-    const int caps[3] = {4096, 8192, capacity_for(HPCTOPK_MAX_K)};
-    for (int c = 0; c < 3; ++c) {
-      int n = 0;
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, main_kernel(), kThreads, smem_bytes_for(caps[c], true)) != cudaSuccess || n < 1) {
-        cudaGetLastError();
-        return HPCTOPK_ERR_CUDA;
+    for (int sp = 0; sp < 2; ++sp)
+      for (int c = 0; c < 3; ++c) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, v.fn, v.threads, smem_bytes_for(class_cap_s(c), sp != 0)) != cudaSuccess || n < 1) {
+          cudaGetLastError();
+          return HPCTOPK_ERR_CUDA;
+        }
+        di.ctas_per_sm[sp][c] = n;
       }
-      di.ctas_per_sm[c] = n;
-    }
     di.ready = true;
   }
+  const Variant& v = kVariants[di.variant];
+  const int cls = cap_class(K);
   Params P;
   P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
   P.num_rows = num_rows; P.K = K; P.out_idx = out_idx; P.out_val = out_val;
   P.ws = static_cast<unsigned char*>(workspace);
-  P.cap = cap; P.stride = stride_for(K);
+  P.cap = capacity_for(K);
+  P.cap_s = class_cap_s(cls) < P.cap ? class_cap_s(cls) : P.cap;
+  P.stride = stride_for(K);
   P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);      // ceil(1.5 K / s)
   P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);      // ceil(1.75 K / s)
   P.split_enabled = split ? 1 : 0;
-  // smem is sized by capacity class so that occupancy (and the grid) depends on K only
-  const int cls = cap_class(cap);
-  const int cls_cap = cls == 0 ? 4096 : (cls == 1 ? 8192 : capacity_for(HPCTOPK_MAX_K));
-  const size_t smem = smem_bytes_for(cls_cap, true);
-  const int grid = di.sm_count * di.ctas_per_sm[cls];
+  const size_t smem = smem_bytes_for(class_cap_s(cls), split);
+  int grid = di.sm_count * di.ctas_per_sm[split ? 1 : 0][cls];
+  if (grid > kMaxGrid) grid = kMaxGrid;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
-  main_kernel()<<<grid, kThreads, smem, st>>>(P);
+  v.fn<<<grid, v.threads, smem, st>>>(P);
   if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
   return HPCTOPK_OK;
 }
