@@ -131,6 +131,35 @@ int hpctopk_read_stats(const void* workspace, hpctopk_stats* host_out, hpctopk_s
 int hpctopk_read_row_info(const void* workspace, int32_t num_rows, hpctopk_row_info* host_out,
                           hpctopk_stream_t stream);
 
+/* Selection for callers that cannot provide a workspace.  (The paper has no counterpart; this
+ * is a convenience of this library.)
+ *
+ * Some callers have no way to obtain device scratch memory at the point where they need a
+ * selection: code that runs inside a framework's allocator-free region (for example while another
+ * component holds the allocator, or in a plug-in that is only handed input and output buffers),
+ * or start-up / shutdown paths where calling cudaMalloc is not allowed or would synchronise the
+ * device.  This entry point takes the same inputs and outputs as hpctopk_select but no workspace:
+ * its scratch is a fixed array of about 10 MB that lives in the library's device image, one copy
+ * on every GPU that loads the library, for the lifetime of the process.  The call itself
+ * allocates nothing and frees nothing.
+ *
+ * Limits: num_rows <= HPCTOPK_STATIC_MAX_ROWS and K <= HPCTOPK_STATIC_MAX_K; anything larger is
+ * rejected with HPCTOPK_ERR_WORKSPACE and nothing is enqueued.  Results are identical to
+ * hpctopk_select (same kernel, possibly a smaller grid).
+ *
+ * The first call on each device resolves the array's device address and caches launch
+ * attributes; make that first call with the device current and before starting any stream
+ * capture.  All calls on a device share the one array: it still holds the previous call's
+ * contents (the call clears the part that must start at zero), and two calls that may overlap
+ * on the GPU (different streams, or a graph replay racing a direct call) would corrupt each
+ * other, so serialise them.  The counters of the last call cannot be read back through
+ * hpctopk_read_stats, which needs a caller workspace. */
+#define HPCTOPK_STATIC_MAX_ROWS 64
+#define HPCTOPK_STATIC_MAX_K 2048
+int hpctopk_select_static(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
+                          int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                          hpctopk_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -60,6 +60,8 @@ def lib():
         L.hpctopk_query_policy.restype = ctypes.c_int
         L.hpctopk_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.hpctopk_select.restype = ctypes.c_int
+        L.hpctopk_select_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+        L.hpctopk_select_static.restype = ctypes.c_int
         L.hpctopk_read_stats.argtypes = [vp, ctypes.POINTER(Stats), vp]
         L.hpctopk_read_stats.restype = ctypes.c_int
         L.hpctopk_read_row_info.argtypes = [vp, i32, vp, vp]
@@ -129,6 +131,36 @@ def hpctopk_select(scores, row_starts, row_lengths, K, out_idx=None, out_val=Non
     if st != HPCTOPK_OK:
         raise HpcTopkError(st)
     return out_idx, out_val, workspace
+
+
+HPCTOPK_STATIC_MAX_ROWS = 64
+HPCTOPK_STATIC_MAX_K = 2048
+
+
+def hpctopk_select_static_raw(scores_ptr, row_starts_ptr, row_lengths_ptr, num_rows, K, out_idx_ptr,
+                              out_val_ptr, stream_ptr):
+    """The workspace-free C entry point on raw addresses; returns the status code."""
+    return int(lib().hpctopk_select_static(scores_ptr, row_starts_ptr, row_lengths_ptr, int(num_rows), int(K),
+                                           out_idx_ptr, out_val_ptr, stream_ptr))
+
+
+def hpctopk_select_static(scores, row_starts, row_lengths, K, out_idx, out_val=None, stream=None):
+    """Select into caller-provided outputs using the library's built-in scratch array.
+
+    For callers that cannot allocate device memory at the call site: nothing is allocated
+    here either, so `out_idx` (and `out_val`, if wanted) must already exist.  At most
+    HPCTOPK_STATIC_MAX_ROWS rows and K <= HPCTOPK_STATIC_MAX_K; calls must not overlap on the GPU.
+    """
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream(scores.device)
+    with torch.cuda.device(scores.device):
+        st = hpctopk_select_static_raw(scores.data_ptr(), row_starts.data_ptr(), row_lengths.data_ptr(),
+                                       int(row_lengths.numel()), K, out_idx.data_ptr(),
+                                       out_val.data_ptr() if out_val is not None else None, stream.cuda_stream)
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    return out_idx, out_val
 
 
 def hpctopk_read_stats(workspace, stream=None):

@@ -961,3 +961,76 @@ int hpctopk_read_row_info(const void* workspace, int32_t num_rows, hpctopk_row_i
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------- selection without a caller workspace
+// Scratch for hpctopk_select_static: one fixed array per GPU that loads the library, held until
+// the process exits.  In host code `g_static_scratch` is only a handle for the runtime; the
+// device address is obtained once per device with cudaGetSymbolAddress and cached below.
+namespace {
+constexpr int kStaticMaxRows = HPCTOPK_STATIC_MAX_ROWS;
+constexpr int kStaticMaxK = HPCTOPK_STATIC_MAX_K;
+constexpr int kStaticMaxGrid = 160;
+constexpr size_t static_layout_bytes(size_t rows, size_t cap, size_t cap_s, size_t grid) {
+  return ((kOffRowInfo + rows * sizeof(hpctopk_row_info) + 255) / 256 * 256)   // control block, counters, row records
+         + (rows < (size_t)kSplitRowsMax ? rows : (size_t)kSplitRowsMax) * cap * 8   // published ranges of split rows
+         + grid * (cap - cap_s) * 8;                                           // overflow slice per CTA
+}
+constexpr size_t kStaticScratchBytes =
+    (static_layout_bytes(kStaticMaxRows, 4 * kStaticMaxK, 2 * kStaticMaxK, kStaticMaxGrid) + 255) / 256 * 256;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+void* g_static_scratch_addr[64] = {nullptr};
+}  // namespace
+
+extern "C" int hpctopk_select_static(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
+                                     int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                                     hpctopk_stream_t stream) {
+  if (num_rows < 0 || K < 1) return HPCTOPK_ERR_INVALID_ARG;
+  if (K > kStaticMaxK || num_rows > kStaticMaxRows) return HPCTOPK_ERR_WORKSPACE;   // beyond the fixed scratch
+  if (num_rows == 0) return HPCTOPK_OK;
+  if (!scores || !row_starts || !row_lengths || !out_idx) return HPCTOPK_ERR_INVALID_ARG;
+  if ((uintptr_t)scores & 15u) return HPCTOPK_ERR_MISALIGNED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HPCTOPK_ERR_CUDA;
+  const Variant& v = kVariants[0];
+  static int sm_count[64] = {0};
+  static int ctas_per_sm[64][3] = {{0}};
+  if (!g_static_scratch_addr[dev]) {
+    // one-time set-up on this device (the device is current): resolve the array's device address
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
+    if (cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
+    if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_for(class_cap_s(2), true)) != cudaSuccess) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    for (int c = 0; c < 3; ++c) {
+      int n = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, v.fn, v.threads, smem_bytes_for(class_cap_s(c), true)) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        return HPCTOPK_ERR_CUDA;
+      }
+      ctas_per_sm[dev][c] = n;
+    }
+    g_static_scratch_addr[dev] = addr;
+  }
+  const int cls = cap_class(K);
+  Params P;
+  P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
+  P.num_rows = num_rows; P.K = K; P.out_idx = out_idx; P.out_val = out_val;
+  P.ws = static_cast<unsigned char*>(g_static_scratch_addr[dev]);
+  P.cap = capacity_for(K);
+  P.cap_s = class_cap_s(cls) < P.cap ? class_cap_s(cls) : P.cap;
+  P.stride = stride_for(K);
+  P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);
+  P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);
+  P.split_enabled = 1;                                   // num_rows <= kStaticMaxRows <= kSplitRowsMax
+  int grid = sm_count[dev] * ctas_per_sm[dev][cls];
+  if (grid > kStaticMaxGrid) grid = kStaticMaxGrid;
+  if (static_layout_bytes((size_t)num_rows, (size_t)P.cap, (size_t)P.cap_s, (size_t)grid) > kStaticScratchBytes) return HPCTOPK_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  // the array keeps the previous call's contents: the control block must start at zero
+  if (cudaMemsetAsync(P.ws, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
+  v.fn<<<grid, v.threads, smem_bytes_for(class_cap_s(cls), true), st>>>(P);
+  if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
+  return HPCTOPK_OK;
+}

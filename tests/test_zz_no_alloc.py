@@ -1,0 +1,51 @@
+"""The workspace-free entry point (hpctopk_select_static) against the regular one.
+
+Some callers cannot allocate device memory where they need a selection (allocator-free
+regions of a framework, plug-ins that only receive buffers, start-up and shutdown paths), so
+the library also offers a call whose scratch is a fixed array inside the library.  This test
+drives it through the C ABI twice in a row, on different inputs, and requires the same
+selection as hpctopk_select, bit for bit (index sets and values); the second call shows that
+the contents left in the shared array by the first do no harm.  It also checks that sizes
+beyond the fixed limits are refused.  The file name makes pytest collect it last.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_08450_b200 import binding as B, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _sorted_pairs(idx, val):
+    order = np.argsort(idx, axis=1, kind="stable")
+    return np.take_along_axis(idx, order, 1), np.take_along_axis(val.view(np.uint32), order, 1)
+
+
+def test_static_scratch_entry_matches_workspace_entry_on_two_calls_in_a_row():
+    from paper_2609_08450_b200 import build
+    build.build()
+    K = 2048
+    batches = [W.config1(DEV, seed=31, num_rows=24, max_len=150000),     # short, direct, sampled and split rows
+               W.config4(DEV, seed=32, num_rows=3, len_lo=300000, len_hi=400000),
+               W.config5(1024, B.hpctopk_query_policy(1024, 65536)[0], DEV, num_rows=64)]
+    for batch, k in zip(batches, (K, K, 1024)):
+        M = batch.num_rows
+        ref_idx, ref_val, _ = B.hpctopk_select(batch.scores, batch.row_starts, batch.row_lengths, k)
+        out_idx = torch.full((M, k), -5, dtype=torch.int32, device=DEV)
+        out_val = torch.zeros((M, k), dtype=torch.float32, device=DEV)
+        B.hpctopk_select_static(batch.scores, batch.row_starts, batch.row_lengths, k, out_idx, out_val)
+        torch.cuda.synchronize()
+        gi, gv = _sorted_pairs(out_idx.cpu().numpy(), out_val.cpu().numpy())
+        ri, rv = _sorted_pairs(ref_idx.cpu().numpy(), ref_val.cpu().numpy())
+        assert np.array_equal(gi, ri) and np.array_equal(gv, rv), batch.name
+
+
+def test_static_scratch_entry_refuses_sizes_beyond_its_limits():
+    p = 0x1000
+    f = B.hpctopk_select_static_raw
+    assert f(p, p, p, B.HPCTOPK_STATIC_MAX_ROWS + 1, 8, p, None, None) == 4
+    assert f(p, p, p, 4, B.HPCTOPK_STATIC_MAX_K + 1, p, None, None) == 4
+    assert f(p, p, p, 0, 8, p, None, None) == 0
+    assert f(None, p, p, 4, 8, p, None, None) == 1
