@@ -20,6 +20,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <stdlib.h>
+#include <type_traits>
 
 #include "../../include/hpctopk.h"
 
@@ -806,6 +807,10 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
   }
 }
 
+}  // namespace
+#include "hpctopk_ws.cuh"
+namespace {
+
 // ---------------------------------------------------------------- host side
 using KernelFn = void (*)(const Params);
 struct Variant {
@@ -821,11 +826,13 @@ const Variant kVariants[] = {
     {hpctopk_kernel<128, 4, 6>, 128},
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
+// 0 selects the warp-specialised kernel, v >= 1 the single-role kernel kVariants[v - 1].
+constexpr int kDefaultVariant = 1;
 
 struct DeviceInfo {
   bool ready = false;
   int sm_count = 0;
-  int variant = 0;
+  int variant = 0;      // 0: warp-specialised kernel; v >= 1: single-role kernel kVariants[v - 1]
   int ctas_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // [split][capacity class]
 };
 DeviceInfo g_dev[64];
@@ -867,7 +874,10 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
   const size_t split_rows = max_num_rows < kSplitRowsMax ? (size_t)max_num_rows : (size_t)kSplitRowsMax;
   size_t b = align_up(kOffRowInfo + (size_t)max_num_rows * sizeof(hpctopk_row_info), 256);
   b += split_rows * cap * 8;                       // published candidate ranges of split rows
-  b += (size_t)kMaxGrid * (cap - cap_s) * 8;       // one overflow slice per resident CTA
+  size_t spill = (size_t)kMaxGrid * (cap - cap_s) * 8;       // one overflow slice per resident CTA
+  const size_t spill_ws = wsk::ws_spill_bytes(K, wsk::kWsMaxGrid);
+  if (spill_ws > spill) spill = spill_ws;
+  b += spill;
   return align_up(b, 256);
 }
 
@@ -896,9 +906,14 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   if (!di.ready) {
     if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
     const char* env = getenv("HPCTOPK_VARIANT");
-    di.variant = env ? atoi(env) : 0;
-    if (di.variant < 0 || di.variant >= kNumVariants) di.variant = 0;
-    const Variant& v = kVariants[di.variant];
+    di.variant = env ? atoi(env) : kDefaultVariant;
+    if (di.variant < 0 || di.variant > kNumVariants) di.variant = kDefaultVariant;
+    if (cudaFuncSetAttribute(wsk::hpctopk_ws_kernel<wsk::kWsU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)wsk::ws_smem_bytes(HPCTOPK_MAX_K, true)) != cudaSuccess) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    const Variant& v = kVariants[di.variant > 0 ? di.variant - 1 : 0];
     const size_t max_smem = smem_bytes_for(class_cap_s(2), true);
     if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
       cudaGetLastError();
@@ -915,7 +930,7 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
       }
     di.ready = true;
   }
-  const Variant& v = kVariants[di.variant];
+  const Variant& v = kVariants[di.variant > 0 ? di.variant - 1 : 0];
   const int cls = cap_class(K);
   Params P;
   P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
@@ -932,7 +947,12 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   if (grid > kMaxGrid) grid = kMaxGrid;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
-  v.fn<<<grid, v.threads, smem, st>>>(P);
+  if (di.variant == 0) {
+    int ws_grid = di.sm_count < wsk::kWsMaxGrid ? di.sm_count : wsk::kWsMaxGrid;
+    wsk::hpctopk_ws_kernel<wsk::kWsU><<<ws_grid, wsk::THREADS, wsk::ws_smem_bytes(K, split), st>>>(P);
+  } else {
+    v.fn<<<grid, v.threads, smem, st>>>(P);
+  }
   if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
   return HPCTOPK_OK;
 }
