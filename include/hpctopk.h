@@ -114,7 +114,9 @@ int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacit
  *   stream      all work is enqueued on `stream` (one small memset and one kernel whose
  *               launch geometry depends only on num_rows, K and the device); nothing is
  *               read back, so the call can be captured in a CUDA graph and replayed with
- *               new contents in the same buffers
+ *               new contents in the same buffers.  The very first call on a device also
+ *               fills a 8 KB lookup table and synchronises the device once: make it
+ *               outside any capture
  *
  * Returns HPCTOPK_OK or an error code; on error nothing was enqueued.  num_rows == 0 is OK. */
 int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
@@ -147,9 +149,9 @@ int hpctopk_read_row_info(const void* workspace, int32_t num_rows, hpctopk_row_i
  * rejected with HPCTOPK_ERR_WORKSPACE and nothing is enqueued.  Results are identical to
  * hpctopk_select (same kernel, possibly a smaller grid).
  *
- * The first call on each device resolves the array's device address and caches launch
- * attributes; make that first call with the device current and before starting any stream
- * capture.  All calls on a device share the one array: it still holds the previous call's
+ * The first call on each device resolves the array's device address, caches launch attributes
+ * and fills a small lookup table (this set-up synchronises the device once); make that first
+ * call with the device current and before starting any stream capture.  All calls on a device share the one array: it still holds the previous call's
  * contents (the call clears the part that must start at zero), and two calls that may overlap
  * on the GPU (different streams, or a graph replay racing a direct call) would corrupt each
  * other, so serialise them.  The counters of the last call cannot be read back through

@@ -33,6 +33,7 @@ class Stats(ctypes.Structure):
                      "cycles_finish", "cycles_total"):
             d[name] = int(getattr(self, name))
         d["cycles_detail"] = [int(v) for v in self.cycles_detail]
+        d["reserved"] = [int(v) for v in self.reserved]
         return d
 
 

@@ -34,6 +34,7 @@ constexpr int kBins = 2048;            // B_c and the widest refinement digit
 constexpr int kSplitRowsMax = 512;     // rows beyond this are never split (enough row parallelism)
 constexpr int kSegMinElems = 16384;    // shortest segment worth a CTA
 constexpr int kTasksPerCta = 2;        // split target: tasks >= kTasksPerCta * grid
+constexpr int kSmallMax = kBins / 2;   // boundary group resolved by direct ranking (pairs held in the histogram's memory)
 
 // workspace layout (bytes)
 constexpr size_t kOffCtrl = 0;                       // uint32 task_counter
@@ -77,16 +78,18 @@ struct Shared {
   uint32_t warp_sums[32];
   uint32_t cand_count;
   uint32_t out_count;
+  uint32_t small_count;
   int32_t loc_bin[2];
   uint32_t loc_below[2];
   uint32_t loc_at[2];
-  uint32_t cutd[2];
+  uint32_t cutd[3];          // cutoffs of tau_0, tau_1 and of the bracket bin tau_hi
   int32_t task;
   int32_t claim;
   uint32_t bcast0;
   uint32_t bcast1;
   uint32_t seg_len_vec;     // vectors per segment unit (split table)
   uint32_t total_tasks;
+  unsigned long long* detail;   // hpctopk_stats::cycles_detail of this call's workspace (tuning aid)
 };
 
 // Dynamic shared memory: [Shared][cand: cap x (kd, idx) pairs][seg_base: kSplitRowsMax + 1 u32].
@@ -130,6 +133,123 @@ __device__ __noinline__ uint32_t cutoff_of_bin(int tau) {
     lo += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, ok)) << sh;
   }
   return lo;
+}
+
+// Bin -> cutoff table: g_cut_table[tau] is the largest descending key whose coarse bin is <= tau
+// (the inclusive FP32 endpoint of Section 5.2).  It depends on the coarse map only, so it is
+// filled once per device by init_cut_table_kernel and read from then on.
+__device__ uint32_t g_cut_table[kBins];
+__global__ void init_cut_table_kernel() {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (warp < kBins) {
+    const uint32_t c = cutoff_of_bin(warp);
+    if ((threadIdx.x & 31) == 0) g_cut_table[warp] = c;
+  }
+}
+
+#define DSTAMP(k, t_prev) do { if (threadIdx.x == 0) { const long long t_now = clock64(); atomicAdd(&SH().detail[k], (unsigned long long)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+
+// ---------------------------------------------------------------- warp-level primitives
+// min{b : H(b) >= quota} over the 2048-bin histogram, by one warp: lane sums of 64 bins, warp
+// prefix, then the 64 bins of the lane that holds the quota are scanned two per lane.
+// Returns the bin (or -1), with H(b - 1) in `below` and h(b) in `at`; uniform across the warp.
+struct LaneSums { uint32_t sum, incl; };
+__device__ __forceinline__ LaneSums w_lane_sums(const uint32_t* hist, int lane) {
+  // lane l owns bins [64 l, 64 l + 64); its sixteen 16-byte chunks are read in an order rotated
+  // by l, so that the lanes of a quarter warp touch different banks
+  const uint4* hv = reinterpret_cast<const uint4*>(hist + lane * 64);
+  uint32_t sum = 0;
+#pragma unroll
+  for (int b = 0; b < 16; ++b) { const uint4 v = hv[(b + lane) & 15]; sum += v.x + v.y + v.z + v.w; }
+  uint32_t incl = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= d) incl += n;
+  }
+  return LaneSums{sum, incl};
+}
+__device__ __forceinline__ int w_locate(const uint32_t* hist, const LaneSums ls, uint32_t quota, int lane,
+                                        uint32_t& below, uint32_t& at) {
+  const uint32_t excl = ls.incl - ls.sum;
+  const uint32_t hit = __ballot_sync(0xFFFFFFFFu, excl < quota && quota <= ls.incl);
+  if (hit == 0u) { below = 0; at = 0; return -1; }
+  const int L = __ffs(hit) - 1;
+  const uint32_t base = __shfl_sync(0xFFFFFFFFu, excl, L);
+  const uint2 pr = *reinterpret_cast<const uint2*>(hist + L * 64 + 2 * lane);
+  const uint32_t s2 = pr.x + pr.y;
+  uint32_t incl2 = s2;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl2, d);
+    if (lane >= d) incl2 += n;
+  }
+  const uint32_t excl2 = base + incl2 - s2;
+  const uint32_t hit2 = __ballot_sync(0xFFFFFFFFu, excl2 < quota && quota <= excl2 + s2);
+  const int M = __ffs(hit2) - 1;               // exists: the quota lies inside lane L's bins
+  const bool first = excl2 + pr.x >= quota;
+  const int bin_m = L * 64 + 2 * lane + (first ? 0 : 1);
+  const uint32_t below_m = first ? excl2 : excl2 + pr.x;
+  const uint32_t at_m = first ? pr.x : pr.y;
+  below = __shfl_sync(0xFFFFFFFFu, below_m, M);
+  at = __shfl_sync(0xFFFFFFFFu, at_m, M);
+  return __shfl_sync(0xFFFFFFFFu, bin_m, M);
+}
+// Three quotas located together: the three dependent chains of shuffles and loads advance in
+// lockstep, so their latencies overlap instead of adding up (a warp issues in order).
+__device__ __forceinline__ void w_locate3(const uint32_t* hist, const LaneSums ls, const uint32_t (&quota)[3], int lane,
+                                          int (&bin)[3]) {
+  const uint32_t excl = ls.incl - ls.sum;
+  uint32_t hit[3];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) hit[k] = __ballot_sync(0xFFFFFFFFu, excl < quota[k] && quota[k] <= ls.incl);
+  int L[3];
+  uint32_t base[3];
+  uint2 pr[3];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) { L[k] = hit[k] ? __ffs(hit[k]) - 1 : 0; base[k] = __shfl_sync(0xFFFFFFFFu, excl, L[k]); }
+#pragma unroll
+  for (int k = 0; k < 3; ++k) pr[k] = *reinterpret_cast<const uint2*>(hist + L[k] * 64 + 2 * lane);
+  uint32_t s2[3], incl2[3];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) { s2[k] = pr[k].x + pr[k].y; incl2[k] = s2[k]; }
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    uint32_t n[3];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) n[k] = __shfl_up_sync(0xFFFFFFFFu, incl2[k], d);
+#pragma unroll
+    for (int k = 0; k < 3; ++k) if (lane >= d) incl2[k] += n[k];
+  }
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    const uint32_t excl2 = base[k] + incl2[k] - s2[k];
+    const uint32_t hit2 = __ballot_sync(0xFFFFFFFFu, excl2 < quota[k] && quota[k] <= excl2 + s2[k]);
+    const int M = hit2 ? __ffs(hit2) - 1 : 0;
+    const int bin_m = L[k] * 64 + 2 * lane + ((excl2 + pr[k].x >= quota[k]) ? 0 : 1);
+    bin[k] = (hit[k] && hit2) ? __shfl_sync(0xFFFFFFFFu, bin_m, M) : -1;
+  }
+}
+__device__ __forceinline__ void w_clear_hist(uint32_t* hist, int lane) {
+  uint4* hv = reinterpret_cast<uint4*>(hist);
+#pragma unroll
+  for (int b = 0; b < 16; ++b) hv[b * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
+}
+// Three bin -> cutoff searches advanced together (see cutoff_of_bin): 32 probes per step each.
+__device__ __forceinline__ void w_cutoffs3(const int (&tau)[3], uint32_t (&cut)[3], int lane) {
+  uint32_t lo[3] = {0u, 0u, 0u};
+#pragma unroll 1
+  for (int b = 27; b >= -3; b -= 5) {
+    const int sh = b < 0 ? 0 : b;
+    const uint32_t nprobe = b < 0 ? 3u : 31u;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      const uint64_t probe = (uint64_t)lo[k] + ((uint64_t)(lane + 1) << sh);
+      const bool ok = (uint32_t)lane < nprobe && probe <= 0xFFFFFFFFull && coarse_bin_of_kd((uint32_t)probe) <= tau[k];
+      lo[k] += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, ok)) << sh;
+    }
+  }
+  cut[0] = lo[0]; cut[1] = lo[1]; cut[2] = lo[2];
 }
 
 // ---------------------------------------------------------------- block primitives
@@ -222,8 +342,9 @@ __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v
   if (i < c.cap_s) CAND()[i] = v; else c.spill[i - c.cap_s] = v;
 }
 
-// Append one admitted score: reserve a slot, store (kd, idx), add to the leading-digit histogram
-// (Eq. "first-exact-hist").  Entries beyond the capacity are counted, not stored.
+// Append one admitted score: reserve a slot, store (kd, idx).  Entries beyond the capacity are
+// counted, not stored.  (The histogram of the refinement digit is built from the compacted
+// on-chip tail right after the pass, see select_adaptive; no second row pass is involved.)
 __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const CandCtx& c) {
   Shared& sh = SH();
   const uint32_t kd = kd_of_bits(u);
@@ -234,9 +355,6 @@ __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const
 #endif
   if (pos < c.cap_s) CAND()[pos] = make_uint2(kd, idx);
   else if (pos < c.cap) c.spill[pos - c.cap_s] = make_uint2(kd, idx);
-#if HPCTOPK_EXPERIMENT == 0
-  atomicAdd(&sh.hist[kd >> 21], 1u);
-#endif
 }
 
 // ---------------------------------------------------------------- Phase 2: the complete-row pass
@@ -292,10 +410,12 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
 #pragma unroll
     for (int j = 0; j < U; ++j) {
       buf[j] = __ldcs(p + j * THREADS);
+#if HPCTOPK_EXPERIMENT == 3
       if (!BAND) {
         const float4* q = p + j * THREADS + PF_VEC;
         if (q < pf_end) asm volatile("prefetch.global.L2 [%0];" ::"l"(q));
       }
+#endif
     }
   };
   auto process_tile = [&](const float4 (&buf)[U], uint32_t ibase) {
@@ -469,6 +589,8 @@ __device__ void record_row(const Params& P, int row, int route, int tau, uint32_
 }
 
 // Phase 1 (Section 4.2): sample view -> coarse histogram -> tau_0, tau_1 -> cutoffs in sh.cutd.
+// A third, tighter bin tau_hi at half the rank K (sample rank ceil(K / 2s)) brackets the K-th
+// score from above; its cutoff sizes the refinement digit of select_adaptive.
 // Returns false when the view cannot support the requested sample ranks.
 template <int THREADS>
 __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_t L, int& tau_pack) {
@@ -476,29 +598,145 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   const int s = P.stride;
   const int bits = 31 - __clz(s);
   const int a = bits ? (int)(__brev((uint32_t)(row & (s - 1))) >> (32 - bits)) : 0;   // pi_s: bit reversal
-  const int64_t n_view = L > a ? (L - a + s - 1) / s : 0;
+  const int64_t n_view = L > a ? ((L - a + s - 1) >> bits) : 0;
   tau_pack = -1;
   if (n_view < P.q1) return false;
+  long long ts = clock64();
   __syncthreads();
   clear_hist<THREADS>(sh);
   __syncthreads();
+  DSTAMP(5, ts);
   const float* __restrict__ rowp = P.scores + g0 + a;
-  for (int64_t t = threadIdx.x; t < n_view; t += THREADS) {
-    const uint32_t kd = kd_of_bits(__float_as_uint(__ldg(rowp + t * s)));
-    atomicAdd(&sh.hist[coarse_bin_of_kd(kd)], 1u);
+  for (int64_t t0 = 0; t0 < n_view; t0 += 4 * THREADS) {
+    uint32_t u[4];
+    bool v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int64_t t = t0 + k * THREADS + threadIdx.x;
+      v[k] = t < n_view;
+      u[k] = v[k] ? __float_as_uint(__ldg(rowp + t * s)) : 0u;
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (v[k]) atomicAdd(&sh.hist[coarse_bin_of_kd(kd_of_bits(u[k]))], 1u);
   }
   __syncthreads();
-  locate<THREADS>(sh, (uint32_t)P.q0, (uint32_t)P.q1, 2);
-  const int tau0 = sh.loc_bin[0], tau1 = sh.loc_bin[1];
-  if (threadIdx.x < 32) {
-    const uint32_t c0 = cutoff_of_bin(tau0);
-    if (threadIdx.x == 0) sh.cutd[0] = c0;
-  } else if (threadIdx.x < 64) {
-    const uint32_t c1 = cutoff_of_bin(tau1);
-    if (threadIdx.x == 32) sh.cutd[1] = c1;
+  DSTAMP(6, ts);
+  if (threadIdx.x < 32) {                       // one warp locates the three bins and looks their cutoffs up
+    const int lane = threadIdx.x;
+    const LaneSums ls = w_lane_sums(sh.hist, lane);
+    uint32_t below, at;
+    int q_hi = (P.K + 2 * s - 1) / (2 * s);
+    if (q_hi < 1) q_hi = 1;
+    const uint32_t quota[3] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi};
+    int tau[3];
+    w_locate3(sh.hist, ls, quota, lane, tau);
+    (void)below; (void)at;
+    if (lane < 3) sh.cutd[lane] = g_cut_table[lane == 0 ? tau[0] : (lane == 1 ? tau[1] : tau[2])];
+    if (lane == 0) { sh.loc_bin[0] = tau[0]; sh.loc_bin[1] = tau[1]; }
   }
   __syncthreads();
-  tau_pack = tau0 | (tau1 << 16);
+  DSTAMP(7, ts);
+  tau_pack = sh.loc_bin[0] | (sh.loc_bin[1] << 16);
+  return true;
+}
+
+// Phase 3 with a row-adaptive first digit (any monotone digit of the key is a valid refinement
+// digit, Section 4.4): d = min((cut_base - kd) >> sh, 2047) measures the distance from the
+// admitted cutoff in units of 2^sh ulps, with sh chosen so that the bracket [cut_hi, cut_base]
+// spans the 2048 bins; only a handful of scores then share the boundary bin.  One histogram pass,
+// one boundary search (every warp for itself), one commit pass; the boundary bin is resolved by
+// ranking its members against each other under (kd, idx).  Returns false, with nothing written,
+// when the K-th score falls outside the bracket or the boundary bin is too large: the caller
+// then runs the general 11+11+10 refinement.
+template <int THREADS>
+__device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint32_t K, uint32_t cut_base, uint32_t cut_hi,
+                                             int32_t* out_idx, float* out_val) {
+  Shared& sh = SH();
+  const int tid = threadIdx.x, lane = tid & 31;
+  const uint32_t span = cut_base > cut_hi ? cut_base - cut_hi : 0u;
+  int shv = 0;
+  while (shv < 31 && (span >> shv) >= 2047u) ++shv;
+  // digit: 0 = the clamped group far above the bracket, 2047 = next to the cutoff
+  auto digit = [&](uint32_t kd) -> uint32_t {
+    const uint32_t d = (cut_base - kd) >> shv;
+    return 2047u - (d < 2047u ? d : 2047u);
+  };
+  long long ts = clock64();
+  __syncthreads();
+  clear_hist<THREADS>(sh);
+  if (tid == 0) { sh.out_count = 0; sh.small_count = 0; }
+  __syncthreads();
+  DSTAMP(0, ts);
+  for (uint32_t i0 = 0; i0 < C; i0 += 4 * THREADS) {
+    uint2 c[4];
+    bool v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { const uint32_t i = i0 + k * THREADS + tid; v[k] = i < C; c[k] = v[k] ? cand_load(cc, i) : make_uint2(0u, 0u); }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) if (v[k]) atomicAdd(&sh.hist[digit(c[k].x)], 1u);
+  }
+  __syncthreads();
+  DSTAMP(1, ts);
+  if (tid < 32) {
+    const LaneSums ls = w_lane_sums(sh.hist, lane);
+    uint32_t below0, at0;
+    const int b0 = w_locate(sh.hist, ls, K, lane, below0, at0);
+    if (lane == 0) { sh.loc_bin[0] = b0; sh.loc_below[0] = below0; sh.loc_at[0] = at0; }
+  }
+  __syncthreads();
+  const int b = sh.loc_bin[0];
+  const uint32_t below = sh.loc_below[0], at = sh.loc_at[0];
+  DSTAMP(2, ts);
+  if (b <= 0 || at > (uint32_t)kSmallMax) return false;
+  const uint32_t k_rem = K - below;             // to take from the boundary bin
+  uint2* const list = reinterpret_cast<uint2*>(sh.hist);
+  __syncthreads();                              // the histogram's memory becomes the boundary list
+  for (uint32_t i0 = 0; i0 < C; i0 += 4 * THREADS) {
+    uint2 c[4];
+    uint32_t dg[4];
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t i = i0 + k * THREADS + tid;
+      c[k] = i < C ? cand_load(cc, i) : make_uint2(0u, 0u);
+      dg[k] = i < C ? digit(c[k].x) : 0xFFFFFFFFu;
+      cnt += dg[k] < (uint32_t)b ? 1u : 0u;
+    }
+    const uint32_t incl = warp_inclusive_scan<THREADS>(cnt);
+    const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    uint32_t base = 0;                          // one reservation of output slots per warp and batch
+    if (lane == 31 && tot) base = atomicAdd(&sh.out_count, tot);
+    base = __shfl_sync(0xFFFFFFFFu, base, 31);
+    uint32_t pos = base + incl - cnt;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (dg[k] < (uint32_t)b) {
+        if (pos < K) { out_idx[pos] = (int32_t)c[k].y; if (out_val) out_val[pos] = __uint_as_float(bits_of_kd(c[k].x)); }
+        ++pos;
+      } else if (dg[k] == (uint32_t)b) {
+        const uint32_t lp = atomicAdd(&sh.small_count, 1u);
+        if (lp < (uint32_t)kSmallMax) list[lp] = c[k];
+      }
+    }
+  }
+  __syncthreads();
+  DSTAMP(3, ts);
+  for (uint32_t i = tid; i < at; i += THREADS) {
+    const uint2 me = list[i];
+    const uint64_t mine = ((uint64_t)me.x << 32) | me.y;
+    uint32_t rank = 0;
+    for (uint32_t t = 0; t < at; ++t) {
+      const uint2 o = list[t];
+      rank += ((((uint64_t)o.x << 32) | o.y) < mine) ? 1u : 0u;
+    }
+    if (rank < k_rem) {
+      out_idx[below + rank] = (int32_t)me.y;
+      if (out_val) out_val[below + rank] = __uint_as_float(bits_of_kd(me.x));
+    }
+  }
+  __syncthreads();
+  DSTAMP(4, ts);
   return true;
 }
 
@@ -534,14 +772,6 @@ __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t
     cfin = C0;
   } else {
     // band extension: append tau_0 < c(x) <= tau_1 and extend the histogram (Eq. "rescue-hist")
-    if (!hist_ready) {
-      __syncthreads();
-      clear_hist<THREADS>(sh);
-      __syncthreads();
-      CandidateSource cs{cc, C0};
-      cs.template for_each<THREADS>([&](bool v, uint32_t kd, uint32_t) { if (v) atomicAdd(&sh.hist[kd >> 21], 1u); });
-      hist_ready = true;
-    }
     __syncthreads();
     scan_range<THREADS, U, true>(P.scores, g0, g0, g0 + L, sh.cutd[0], sh.cutd[1], cc);
     __syncthreads();
@@ -552,8 +782,15 @@ __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t
     else route = HPCTOPK_ROUTE_RECOVERY;
   }
   if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND) {
-    CandidateSource cs{cc, cfin};
-    select_and_emit<THREADS>(cs, K, hist_ready, oi, ov);
+    const uint32_t cut_base = route == HPCTOPK_ROUTE_BAND ? sh.cutd[1] : sh.cutd[0];
+    if (!select_adaptive<THREADS>(cc, cfin, K, cut_base, sh.cutd[2], oi, ov)) {
+      if (threadIdx.x == 0) add64(&stats_of(P.ws)->reserved[0], 1);      // general refinement taken
+      __syncthreads();
+      clear_hist<THREADS>(sh);
+      __syncthreads();
+      CandidateSource cs{cc, cfin};
+      select_and_emit<THREADS>(cs, K, false, oi, ov);
+    }
   } else {
     RowSource rs{P.scores, g0, g0 + L};
     select_and_emit<THREADS>(rs, K, false, oi, ov);
@@ -587,7 +824,7 @@ __device__ void process_row(const Params& P, int row) {
     scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, 0xFFFFFFFFu, cc);
     __syncthreads();
     CandidateSource cs{cc, (uint32_t)L};
-    select_and_emit<THREADS>(cs, K, true, oi, ov);
+    select_and_emit<THREADS>(cs, K, false, oi, ov);
     record_row(P, row, HPCTOPK_ROUTE_DIRECT, -1, (uint32_t)L, (uint32_t)L, (uint64_t)L, 0, (uint64_t)L);
     return;
   }
@@ -725,6 +962,8 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
   uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl);
   const int tid = threadIdx.x;
 
+  if (tid == 0) sh.detail = reinterpret_cast<unsigned long long*>(P.ws + kOffStats + offsetof(hpctopk_stats, cycles_detail));
+  __syncthreads();
   uint32_t total_tasks = (uint32_t)P.num_rows;
   if (P.split_enabled) {
     // Device-side ragged dispatch: every CTA derives the same task table from row_lengths.
@@ -808,6 +1047,12 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
 }
 
 }  // namespace
+#include "hpctopk_ws.cuh"            // namespace wsk: scanner warps + helper groups
+#define HPCTOPK_WS_NAMESPACE wsf     // namespace wsf: single-role variant, warp-synchronous compaction
+#define HPCTOPK_WS_FUSED 1
+#define HPCTOPK_NS 16
+#define HPCTOPK_WS_U 2
+#define HPCTOPK_WS_MINB 2
 #include "hpctopk_ws.cuh"
 namespace {
 
@@ -823,11 +1068,14 @@ const Variant kVariants[] = {
     {hpctopk_kernel<512, 2, 2>, 512},
     {hpctopk_kernel<256, 2, 4>, 256},
     {hpctopk_kernel<256, 4, 3>, 256},
-    {hpctopk_kernel<128, 4, 6>, 128},
+    {hpctopk_kernel<512, 2, 3>, 512},
+    {hpctopk_kernel<384, 2, 4>, 384},
+    {hpctopk_kernel<640, 2, 2>, 640},
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 // 0 selects the warp-specialised kernel, v >= 1 the single-role kernel kVariants[v - 1].
 constexpr int kDefaultVariant = 1;
+constexpr int kFusedVariant = 100;     // single-role kernel with warp-synchronous compaction (namespace wsf)
 
 struct DeviceInfo {
   bool ready = false;
@@ -877,6 +1125,8 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
   size_t spill = (size_t)kMaxGrid * (cap - cap_s) * 8;       // one overflow slice per resident CTA
   const size_t spill_ws = wsk::ws_spill_bytes(K, wsk::kWsMaxGrid);
   if (spill_ws > spill) spill = spill_ws;
+  const size_t spill_wf = wsf::ws_spill_bytes(K, kMaxGrid);
+  if (spill_wf > spill) spill = spill_wf;
   b += spill;
   return align_up(b, 256);
 }
@@ -905,15 +1155,22 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   const bool split = num_rows <= kSplitRowsMax;
   if (!di.ready) {
     if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
+    init_cut_table_kernel<<<kBins * 32 / 256, 256>>>();
+    if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
     const char* env = getenv("HPCTOPK_VARIANT");
     di.variant = env ? atoi(env) : kDefaultVariant;
-    if (di.variant < 0 || di.variant > kNumVariants) di.variant = kDefaultVariant;
+    if (di.variant != kFusedVariant && (di.variant < 0 || di.variant > kNumVariants)) di.variant = kDefaultVariant;
     if (cudaFuncSetAttribute(wsk::hpctopk_ws_kernel<wsk::kWsU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)wsk::ws_smem_bytes(HPCTOPK_MAX_K, true)) != cudaSuccess) {
       cudaGetLastError();
       return HPCTOPK_ERR_CUDA;
     }
-    const Variant& v = kVariants[di.variant > 0 ? di.variant - 1 : 0];
+    if (cudaFuncSetAttribute(wsf::hpctopk_ws_kernel<wsf::kWsU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)wsf::ws_smem_bytes(HPCTOPK_MAX_K, true)) != cudaSuccess) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    const Variant& v = kVariants[(di.variant > 0 && di.variant <= kNumVariants) ? di.variant - 1 : 0];
     const size_t max_smem = smem_bytes_for(class_cap_s(2), true);
     if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
       cudaGetLastError();
@@ -930,7 +1187,7 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
       }
     di.ready = true;
   }
-  const Variant& v = kVariants[di.variant > 0 ? di.variant - 1 : 0];
+  const Variant& v = kVariants[(di.variant > 0 && di.variant <= kNumVariants) ? di.variant - 1 : 0];
   const int cls = cap_class(K);
   Params P;
   P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
@@ -947,7 +1204,17 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   if (grid > kMaxGrid) grid = kMaxGrid;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
-  if (di.variant == 0) {
+  if (di.variant == kFusedVariant) {
+    const size_t fsmem = wsf::ws_smem_bytes(K, split);
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wsf::hpctopk_ws_kernel<wsf::kWsU>, wsf::THREADS, fsmem) != cudaSuccess || per_sm < 1) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    int fgrid = di.sm_count * per_sm;
+    if (fgrid > kMaxGrid) fgrid = kMaxGrid;
+    wsf::hpctopk_ws_kernel<wsf::kWsU><<<fgrid, wsf::THREADS, fsmem, st>>>(P);
+  } else if (di.variant == 0) {
     int ws_grid = di.sm_count < wsk::kWsMaxGrid ? di.sm_count : wsk::kWsMaxGrid;
     wsk::hpctopk_ws_kernel<wsk::kWsU><<<ws_grid, wsk::THREADS, wsk::ws_smem_bytes(K, split), st>>>(P);
   } else {
@@ -1018,6 +1285,8 @@ extern "C" int hpctopk_select_static(const float* scores, const int32_t* row_sta
     // one-time set-up on this device (the device is current): resolve the array's device address
     void* addr = nullptr;
     if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
+    init_cut_table_kernel<<<kBins * 32 / 256, 256>>>();      // bin -> cutoff table used by Phase 1
+    if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
     if (cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
     if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_for(class_cap_s(2), true)) != cudaSuccess) {
       cudaGetLastError();

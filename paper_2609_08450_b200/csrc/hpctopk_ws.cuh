@@ -12,30 +12,43 @@
 // it (mbarrier `scanned`), the helpers retire it and post the slot's next task.  A band
 // extension (Eq. "rescue-band") is just another task on the same slot that appends to the
 // same buffer.  Every wait is bounded: on a timeout the CTA raises an error flag and leaves.
-#pragma once
+// The header can be included more than once with different settings (macros below) and a
+// different namespace: HPCTOPK_WS_FUSED = 1 builds the single-role variant in which all warps
+// of the CTA scan a row together and then act as one helper group for the same row.
+#ifndef HPCTOPK_WS_NAMESPACE
+#define HPCTOPK_WS_NAMESPACE wsk
+#endif
+#ifndef HPCTOPK_WS_FUSED
+#define HPCTOPK_WS_FUSED 0
+#endif
+#ifndef HPCTOPK_WS_MINB
+#define HPCTOPK_WS_MINB 1
+#endif
 
-namespace wsk {
+namespace HPCTOPK_WS_NAMESPACE {
 
 #ifndef HPCTOPK_NS
-#define HPCTOPK_NS 28
+#define HPCTOPK_NS 24
 #endif
 #ifndef HPCTOPK_GROUPS
 #define HPCTOPK_GROUPS 4
 #endif
 #ifndef HPCTOPK_GW
-#define HPCTOPK_GW 1
+#define HPCTOPK_GW 2
 #endif
 #ifndef HPCTOPK_WS_U
 #define HPCTOPK_WS_U 4
 #endif
-constexpr int NS = HPCTOPK_NS;         // scanner warps
-constexpr int kSlots = HPCTOPK_GROUPS; // task slots = helper groups (group g owns slot g)
-constexpr int kGW = HPCTOPK_GW;        // warps per helper group
-constexpr int NH = kSlots * kGW;       // helper warps
+constexpr bool kFused = HPCTOPK_WS_FUSED != 0;
+constexpr int NS = HPCTOPK_NS;         // scanner warps (= candidate regions per buffer)
+constexpr int kSlots = kFused ? 1 : HPCTOPK_GROUPS;   // task slots = helper groups (group g owns slot g)
+constexpr int kGW = kFused ? NS : HPCTOPK_GW;         // warps per helper group
+constexpr int NH = kFused ? 0 : kSlots * kGW;         // dedicated helper warps
 constexpr int kWsU = HPCTOPK_WS_U;     // float4 loads per thread per register tile
 constexpr int ST = NS * 32;            // scanner threads
 constexpr int HT = kGW * 32;           // threads per helper group
 constexpr int THREADS = ST + NH * 32;
+constexpr int kMinBlocks = HPCTOPK_WS_MINB;
 constexpr int kSmallMax = kBins / 2;   // frontier size resolved by direct ranking (pairs held in the histogram's memory)
 constexpr int kWsTasksPerCta = 8;      // split target: tasks >= kWsTasksPerCta * grid
 constexpr int kWsMaxGrid = 160;        // CTAs (one per SM) the overflow region is sized for
@@ -48,7 +61,7 @@ struct __align__(16) HelperShared {   // private to one helper group
   int32_t loc_bin[2];
   uint32_t loc_below[2];
   uint32_t loc_at[2];
-  uint32_t cutd[2];
+  uint32_t cutd[4];
   uint32_t bcast0, bcast1;
   int32_t claim;
   int32_t pad;
@@ -60,7 +73,8 @@ struct Grp {
   int g, t;
   __device__ __forceinline__ int tid() const { return t; }
   __device__ __forceinline__ void sync() const {
-    if (HT == 32) __syncwarp();
+    if (kFused) __syncthreads();
+    else if (HT == 32) __syncwarp();
     else asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(HT) : "memory");
   }
 };
@@ -115,6 +129,7 @@ __device__ __noinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity)
     asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
                  : "=r"(ok) : "r"(addr), "r"(parity), "r"(2000u) : "memory");
     if (ok) return true;
+    __nanosleep(400);                      // a poller must not compete with the working warps for issue slots
     if (*reinterpret_cast<volatile int32_t*>(&sh.abort)) return false;
     if ((it & 255u) == 255u) {
       unsigned long long now;
@@ -586,6 +601,211 @@ __device__ __forceinline__ void g_prefetch_row(const Grp& G, const Params& P, in
     asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
 }
 
+
+// ---------------------------------------------------------------- single-warp helper routines
+// A helper warp works alone, so its routines are warp-synchronous: no block barriers, results
+// passed through shuffles, loads issued in batches so that their latencies overlap.
+
+// Phase 1 (Section 4.2) by one warp.  Besides tau_0 and tau_1 it locates a tighter bin tau_hi
+// at half the rank K (sample rank ceil(K / 2s)); its cutoff brackets the K-th score from above
+// and sizes the refinement digit of w_select_adaptive.  Results are uniform across the warp.
+struct Phase1Out { bool usable; int tau_pack; uint32_t cut0, cut1, cut_hi; };
+__device__ __noinline__ Phase1Out w_phase1(const Grp G, const Params& P, int row, int64_t g0, int64_t L) {
+  HelperShared& sh = WSH().h[G.g];
+  const int lane = G.tid() & 31, wi = G.tid() >> 5;     // lane and warp index inside the group
+  Phase1Out o{false, -1, 0u, 0u, 0u};
+  const int s = P.stride;
+  const int bits = 31 - __clz(s);
+  const int a = bits ? (int)(__brev((uint32_t)(row & (s - 1))) >> (32 - bits)) : 0;
+  const int64_t n_view = L > a ? ((L - a + s - 1) >> bits) : 0;
+  if (n_view < P.q1) return o;
+  long long ts = clock64();
+  G.sync();
+  if (wi == 0) w_clear_hist(sh.hist, lane);
+  G.sync();
+  const float* __restrict__ rowp = P.scores + g0 + a;
+  // wide batches: while the scanner warps keep the load/store queues full, every dependent
+  // round trip through them is expensive, so as many loads as possible share one trip
+  for (int64_t t0 = (int64_t)wi * 512; t0 < n_view; t0 += 512 * kGW) {
+    uint32_t u[16];
+    bool v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int64_t t = t0 + k * 32 + lane;
+      v[k] = t < n_view;
+      u[k] = v[k] ? __float_as_uint(__ldg(rowp + t * s)) : 0u;
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k)
+      if (v[k]) atomicAdd(&sh.hist[coarse_bin_of_kd(kd_of_bits(u[k]))], 1u);
+  }
+  G.sync();
+  WSTAMP(1, ts);
+  if (wi == 0) {                                // one warp locates the bins and looks the cutoffs up
+    const LaneSums ls = w_lane_sums(sh.hist, lane);
+    uint32_t below, at;
+    int q_hi = (P.K + 2 * s - 1) / (2 * s);
+    if (q_hi < 1) q_hi = 1;
+    const uint32_t quota[3] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi};
+    int tau[3];
+    w_locate3(sh.hist, ls, quota, lane, tau);
+    (void)below; (void)at;
+    if (lane < 3) sh.cutd[lane] = g_cut_table[lane == 0 ? tau[0] : (lane == 1 ? tau[1] : tau[2])];
+    if (lane == 0) { sh.loc_bin[0] = tau[0]; sh.loc_bin[1] = tau[1]; }
+  }
+  G.sync();
+  WSTAMP(3, ts);
+  o.usable = true;
+  o.tau_pack = sh.loc_bin[0] | (sh.loc_bin[1] << 16);
+  o.cut0 = sh.cutd[0]; o.cut1 = sh.cutd[1]; o.cut_hi = sh.cutd[2];
+  G.sync();                                     // values are in registers before the next row overwrites them
+  return o;
+}
+
+// Phase 3 by one warp over a slot's buffer, with a row-adaptive first digit (any monotone digit
+// of the key is a valid refinement digit, Section 4.4): d = min((cut_base - kd) >> sh, 2047)
+// measures the distance from the admitted cutoff in units of 2^sh ulps; `sh` is chosen so that
+// the bracket [cut_hi, cut_base] spans the 2048 bins, which leaves only a handful of scores
+// in the boundary bin.  One histogram pass, one boundary search, one commit pass; the boundary
+// bin is resolved by ranking its members against each other under (kd, idx).  Returns false
+// (nothing written) when the K-th score falls outside the bracket or the boundary bin is too
+// large; the caller then runs the general 11+11+10 refinement.
+__device__ __noinline__ bool w_select_adaptive(const Grp G, const Buf buf, bool spilled, uint32_t K, uint32_t cut_base,
+                                               uint32_t cut_hi, int32_t* out_idx, float* out_val) {
+  HelperShared& sh = WSH().h[G.g];
+  const int lane = G.tid() & 31, wi = G.tid() >> 5;     // lane and warp index inside the group
+  long long ts = clock64();
+  const uint32_t span = cut_base > cut_hi ? cut_base - cut_hi : 0u;
+  int shv = 0;
+  while (shv < 31 && (span >> shv) >= 2047u) ++shv;
+  G.sync();
+  if (wi == 0) w_clear_hist(sh.hist, lane);
+  if (G.tid() == 0) { sh.small_count = 0; sh.out_count = 0; }
+  G.sync();
+  // digit: 0 = the clamped group far above the bracket, 2047 = next to the cutoff
+  auto digit = [&](uint32_t kd) -> uint32_t {
+    const uint32_t d = (cut_base - kd) >> shv;
+    return 2047u - (d < 2047u ? d : 2047u);
+  };
+  // The filled parts of the NS regions are visited as one flat index space, sixteen entries
+  // per lane and batch (one trip through the shared-memory queue per batch).  Lane w keeps
+  // the fill count of region w; the others obtain it by shuffle.
+  const uint32_t cnt_l = lane < NS ? min(buf.cnt[lane], buf.rw) : 0u;
+  uint32_t jmax = cnt_l;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) jmax = max(jmax, __shfl_xor_sync(0xFFFFFFFFu, jmax, d));
+  const uint32_t jr = (jmax + 31u) & ~31u;
+  const uint32_t total = jr * NS;
+  const uint32_t inv = jr ? (0xFFFFFFFFu / jr + 1u) : 0u;   // w = i / jr for i < 2^16
+  auto fetch = [&](uint32_t i, uint2& c) -> bool {
+    const uint32_t w = min(__umulhi(i, inv), (uint32_t)(NS - 1)), j = i - w * jr;
+    const uint32_t n_w = __shfl_sync(0xFFFFFFFFu, cnt_l, (int)w);
+    const bool v = i < total && j < n_w;
+    c = v ? buf.region0[w * buf.rw + j] : make_uint2(0u, 0u);
+    return v;
+  };
+  // pass A: histogram of the digit (batches dealt to the warps of the group)
+  for (uint32_t i0 = (uint32_t)wi * 512u; i0 < total; i0 += 512u * kGW) {
+    uint2 c[16];
+    bool v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = fetch(i0 + k * 32 + lane, c[k]);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) if (v[k]) atomicAdd(&sh.hist[digit(kd_of_bits(c[k].x))], 1u);
+  }
+  if (spilled) {                                // entries in the overflow slice (uncommon)
+    const uint32_t n_g = (uint32_t)NS << buf.sw_log2;
+    for (uint32_t i = G.tid(); i < n_g; i += Grp::N) {
+      const uint32_t w = i >> buf.sw_log2, j = i & (buf.sw - 1);
+      if (buf.rw + j < buf.cnt[w]) atomicAdd(&sh.hist[digit(kd_of_bits(__ldcg(buf.spill + i).x))], 1u);
+    }
+  }
+  G.sync();
+  if (wi == 0) {                                // one warp locates the boundary bin
+    const LaneSums ls = w_lane_sums(sh.hist, lane);
+    uint32_t below0, at0;
+    const int b0 = w_locate(sh.hist, ls, K, lane, below0, at0);
+    if (lane == 0) { sh.loc_bin[0] = b0; sh.loc_below[0] = below0; sh.loc_at[0] = at0; }
+  }
+  G.sync();
+  const int b = sh.loc_bin[0];
+  const uint32_t below = sh.loc_below[0], at = sh.loc_at[0];
+  WSTAMP(4, ts);
+  if (b <= 0 || at > (uint32_t)kSmallMax) return false;
+  const uint32_t k_rem = K - below;             // to take from the boundary bin
+  uint2* const list = reinterpret_cast<uint2*>(sh.hist);
+  G.sync();                                     // the histogram's memory becomes the boundary list
+  // pass B: commit everything ahead of the boundary bin, collect the boundary bin
+  for (uint32_t i0 = (uint32_t)wi * 512u; i0 < total; i0 += 512u * kGW) {
+    uint2 c[16];
+    uint32_t sel = 0, bnd = 0, cnt = 0;         // bit k: entry k is committed / lies in the boundary bin
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const bool v = fetch(i0 + k * 32 + lane, c[k]);
+      const uint32_t dg = v ? digit(kd_of_bits(c[k].x)) : 0xFFFFFFFFu;
+      if (dg < (uint32_t)b) { sel |= 1u << k; ++cnt; }
+      else if (dg == (uint32_t)b) bnd |= 1u << k;
+    }
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t m = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= d) incl += m;
+    }
+    const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    uint32_t out_base = 0;                      // one reservation of output slots per warp and batch
+    if (lane == 31 && tot) out_base = atomicAdd(&sh.out_count, tot);
+    out_base = __shfl_sync(0xFFFFFFFFu, out_base, 31);
+    uint32_t pos = out_base + incl - cnt;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if ((sel >> k) & 1u) {
+        if (pos < K) { out_idx[pos] = (int32_t)c[k].y; if (out_val) out_val[pos] = __uint_as_float(c[k].x); }
+        ++pos;
+      } else if ((bnd >> k) & 1u) {
+        const uint32_t lp = atomicAdd(&sh.small_count, 1u);
+        if (lp < (uint32_t)kSmallMax) list[lp] = make_uint2(kd_of_bits(c[k].x), c[k].y);
+      }
+    }
+  }
+  if (spilled) {
+    const uint32_t n_g = (uint32_t)NS << buf.sw_log2;
+    for (uint32_t i = G.tid(); i < n_g; i += Grp::N) {
+      const uint32_t w = i >> buf.sw_log2, j = i & (buf.sw - 1);
+      if (buf.rw + j < buf.cnt[w]) {
+        const uint2 c = __ldcg(buf.spill + i);
+        const uint32_t dg = digit(kd_of_bits(c.x));
+        if (dg < (uint32_t)b) {
+          const uint32_t pos = atomicAdd(&sh.out_count, 1u);
+          if (pos < K) { out_idx[pos] = (int32_t)c.y; if (out_val) out_val[pos] = __uint_as_float(c.x); }
+        } else if (dg == (uint32_t)b) {
+          const uint32_t lp = atomicAdd(&sh.small_count, 1u);
+          if (lp < (uint32_t)kSmallMax) list[lp] = make_uint2(kd_of_bits(c.x), c.y);
+        }
+      }
+    }
+  }
+  G.sync();
+  // boundary bin: rank under (kd, idx); the k_rem best are committed
+  for (uint32_t i = G.tid(); i < at; i += Grp::N) {
+    const uint2 me = list[i];
+    const uint64_t mine = ((uint64_t)me.x << 32) | me.y;
+    uint32_t rank = 0;
+    for (uint32_t t = 0; t < at; ++t) {
+      const uint2 o = list[t];
+      rank += ((((uint64_t)o.x << 32) | o.y) < mine) ? 1u : 0u;
+    }
+    if (rank < k_rem) {
+      const uint32_t pos = below + rank;
+      out_idx[pos] = (int32_t)me.y;
+      if (out_val) out_val[pos] = __uint_as_float(bits_of_kd(me.x));
+    }
+  }
+  G.sync();
+  WSTAMP(5, ts);
+  return true;
+}
+
 // ---------------------------------------------------------------- per-slot task state (helper registers)
 struct Task {
   int32_t row, seg, nseg;
@@ -594,6 +814,7 @@ struct Task {
   int32_t tau_pack;
   int32_t banded;        // the band extension has been appended already
   uint32_t cut0, cut1;   // cutoffs of tau_0 and tau_1 (descending keys)
+  uint32_t cut_hi;       // cutoff of the bracket bin at half the rank (sizes the refinement digit)
   uint32_t c0;           // C(tau_0)
   uint64_t scanned, sampled;
   long long t_post;
@@ -618,7 +839,7 @@ __device__ __forceinline__ Buf make_slot_buf(const Params& P, int slot, uint32_t
 template <int U>
 __device__ __noinline__ void scanner_main(const Params& P, uint32_t rw, uint32_t sw) {
   WsShared& sh = WSH();
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = (int)threadIdx.x - NH * 32, warp = tid >> 5, lane = tid & 31;   // helpers hold the lowest warp ids
   uint32_t parity = 0;                    // bit s: parity of the next descriptor of slot s
   uint32_t done = 0;                      // bit s: slot s has posted DONE
   int live = kSlots;
@@ -673,6 +894,20 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
   G.sync();
 
   auto post = [&](int mode, int64_t g0, int64_t e0, int64_t e1, uint32_t cut_lo, uint32_t cut_hi) {
+    if (kFused) {
+      // single-role variant: the group scans the range itself, right now
+      if (mode == MODE_DONE) return;
+      const int warp = ht >> 5;
+      G.sync();
+      if (mode == MODE_SCAN && ht < 32) wsh.cnt[s][ht] = 0;
+      G.sync();
+      uint32_t wbase = wsh.cnt[s][warp];
+      if (mode == MODE_SCAN) wbase = scan_share<ST, kWsU, false>(P.scores, g0, e0, e1, cut_lo, cut_hi, buf, ht, (uint32_t)warp, wbase);
+      else wbase = scan_share<ST, kWsU, true>(P.scores, g0, e0, e1, cut_lo, cut_hi, buf, ht, (uint32_t)warp, wbase);
+      if ((ht & 31) == 0) wsh.cnt[s][warp] = wbase;
+      G.sync();
+      return;
+    }
     if (ht == 0) {
       Desc& d = wsh.desc[s];
       d.g0 = g0; d.e0 = e0; d.e1 = e1; d.cut_lo = cut_lo; d.cut_hi = cut_hi; d.mode = mode;
@@ -712,7 +947,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
       int64_t L = P.row_lengths[row];
       if (L < 0) L = 0;
       t.row = row; t.seg = seg; t.nseg = nseg; t.g0 = g0; t.L = L;
-      t.banded = 0; t.tau_pack = -1; t.c0 = 0; t.scanned = 0; t.sampled = 0; t.cut0 = 0; t.cut1 = 0;
+      t.banded = 0; t.tau_pack = -1; t.c0 = 0; t.scanned = 0; t.sampled = 0; t.cut0 = 0; t.cut1 = 0; t.cut_hi = 0;
       oi = P.out_idx + (int64_t)row * P.K;
       ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
       if (ht == 0) add64(&stats_of(P.ws)->tasks, 1);
@@ -727,7 +962,9 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
         return true;
       }
       const long long t0 = clock64();
-      const bool usable = g_phase1(G, P, row, g0, L, t.tau_pack);
+      const Phase1Out p1 = w_phase1(G, P, row, g0, L);
+      const bool usable = p1.usable;
+      t.tau_pack = p1.tau_pack;
       if (ht == 0) add64(&stats_of(P.ws)->cycles_phase1, (uint64_t)(clock64() - t0));
       t.sampled = usable ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
       if (!usable && nseg == 1) { recover_row(HPCTOPK_ROUTE_RECOVERY, 0, 0); continue; }
@@ -741,8 +978,9 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
         if (e1 < e0) e1 = e0;
         if (!usable) e1 = e0;                      // nothing to scan; the finisher recovers the row
       }
-      t.cut0 = usable ? sh.cutd[0] : 0u;
-      t.cut1 = usable ? sh.cutd[1] : 0u;
+      t.cut0 = p1.cut0;
+      t.cut1 = p1.cut1;
+      t.cut_hi = p1.cut_hi;
       t.e0 = e0; t.e1 = e1; t.t_post = clock64();
       t.scanned = (uint64_t)(e1 - e0);
       post(MODE_SCAN, g0, e0, e1, 0u, t.cut0);
@@ -804,8 +1042,13 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
     } else if (ty.overflow || ty.total > (uint32_t)P.cap) {
       recover_row(HPCTOPK_ROUTE_OVERFLOW, t.c0, t.scanned);
     } else if (ty.total >= K) {
-      BufSource bs{buf, ty.spilled};
-      g_select_and_emit(G, bs, K, oi, ov);
+      bool done = false;
+      done = w_select_adaptive(G, buf, ty.spilled, K, t.banded ? t.cut1 : t.cut0, t.cut_hi, oi, ov);
+      if (!done) {
+        if (ht == 0) add64(&stats_of(P.ws)->reserved[0], 1);      // general refinement taken
+        BufSource bs{buf, ty.spilled};
+        g_select_and_emit(G, bs, K, oi, ov);
+      }
       g_record_row(G, P, t.row, t.banded ? HPCTOPK_ROUTE_BAND : HPCTOPK_ROUTE_PRIMARY, t.tau_pack, t.c0, ty.total,
                    t.scanned, t.sampled, (uint64_t)t.L);
     } else if (!t.banded) {
@@ -824,11 +1067,13 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
 
   bool busy = start_next();
   while (busy) {
-    if (ht == 0) sh.bcast0 = mbar_wait(&wsh.scanned[s], (uses - 1) & 1u) ? 1u : 0u;
-    G.sync();
-    const bool ok = sh.bcast0 != 0u;
-    G.sync();
-    if (!ok) break;
+    if (!kFused) {
+      if (ht == 0) sh.bcast0 = mbar_wait(&wsh.scanned[s], (uses - 1) & 1u) ? 1u : 0u;
+      G.sync();
+      const bool ok = sh.bcast0 != 0u;
+      G.sync();
+      if (!ok) break;
+    }
     if (complete()) busy = start_next();
   }
   post(MODE_DONE, 0, 0, 0, 0u, 0u);       // releases the scanners from this slot
@@ -836,7 +1081,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
 }
 
 template <int U>
-__global__ void __launch_bounds__(THREADS, 1) hpctopk_ws_kernel(const Params P) {
+__global__ void __launch_bounds__(THREADS, kMinBlocks) hpctopk_ws_kernel(const Params P) {
   WsShared& sh = WSH();
   const int tid = threadIdx.x;
   const uint32_t rw = (uint32_t)ws_region_entries(P.K);
@@ -884,12 +1129,19 @@ __global__ void __launch_bounds__(THREADS, 1) hpctopk_ws_kernel(const Params P) 
     total_tasks = sh.total_tasks;
   }
 
-  if (tid < ST) {
+  // The helper groups take the lowest warp ids: the warp schedulers favour older warps, and the
+  // helpers' short, latency-bound phases must not queue behind the streaming warps.
+  if (kFused) {
+    Grp G;
+    G.g = 0;
+    G.t = tid;
+    helper_main(G, P, rw, sw, total_tasks, seg_base);
+  } else if (tid >= NH * 32) {
     scanner_main<U>(P, rw, sw);
   } else {
     Grp G;
-    G.g = (tid - ST) / HT;
-    G.t = (tid - ST) % HT;
+    G.g = tid / HT;
+    G.t = tid % HT;
     helper_main(G, P, rw, sw, total_tasks, seg_base);
   }
 }
@@ -904,4 +1156,13 @@ inline size_t ws_spill_bytes(int K, int grid) {
   return (size_t)grid * kSlots * NS * ws_region_total(K) * 8;
 }
 
-}  // namespace wsk
+}  // namespace HPCTOPK_WS_NAMESPACE
+
+#undef HPCTOPK_WS_NAMESPACE
+#undef HPCTOPK_WS_FUSED
+#undef HPCTOPK_WS_MINB
+#undef HPCTOPK_NS
+#undef HPCTOPK_GROUPS
+#undef HPCTOPK_GW
+#undef HPCTOPK_WS_U
+#undef WSTAMP
