@@ -17,7 +17,6 @@ import json
 import os
 import subprocess
 import sys
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -31,7 +30,7 @@ K = 2048
 # DRAM bytes per score element of the dominant kernel, from the ncu capture summarised in
 # profiles/hpctopk_kernel_config3_small.md (dram__bytes_read.sum + dram__bytes_write.sum over
 # the valid elements of the captured launch; traffic grows in proportion to the elements).
-NCU_DRAM_BYTES_PER_ELEMENT = None
+NCU_DRAM_BYTES_PER_ELEMENT = 4.49
 
 
 def load_peaks():
@@ -43,7 +42,8 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    """Samples SM clocks and throttle reasons with one streaming nvidia-smi process while a
+    region runs (a sample every 20 ms)."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -51,29 +51,35 @@ class ClockSampler:
     def __init__(self, index):
         self.index = index
         self.rows = []
-        self._stop = threading.Event()
-        self._thread = None
-
-    def _run(self):
-        while not self._stop.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
-                parts = [p.strip() for p in out.stdout.strip().split(",")]
-                if len(parts) >= 6:
-                    self.rows.append(parts)
-            except Exception:
-                pass
-            self._stop.wait(0.1)
+        self.proc = None
 
     def __enter__(self):
-        self._thread = threading.Thread(target=self._run, daemon=True)
-        self._thread.start()
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            time.sleep(0.3)          # let the sampler start before the timed region
+        except Exception:
+            self.proc = None
+        self.t0 = time.time()
         return self
 
     def __exit__(self, *a):
-        self._stop.set()
-        self._thread.join(timeout=10)
+        self.t1 = time.time()
+        if self.proc is None:
+            return
+        time.sleep(0.05)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        lines = [l for l in out.strip().splitlines() if l.count(",") >= 5]
+        # keep the samples taken during the region (the sampler started ~0.3 s earlier)
+        total = max(self.t1 - self.t0 + 0.35, 1e-3)
+        keep = max(1, int(round(len(lines) * (self.t1 - self.t0 + 0.05) / total)))
+        self.rows = [[p.strip() for p in l.split(",")] for l in lines[-keep:]]
 
     def summary(self):
         if not self.rows:
@@ -157,8 +163,8 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config3", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--e2e-steps", type=int, default=3)
