@@ -43,7 +43,10 @@ enum {
   HPCTOPK_ROUTE_PRIMARY = 2,  /* C(tau_0) >= K: certified by the primary boundary */
   HPCTOPK_ROUTE_BAND = 3,     /* C(tau_0) < K <= C(tau_1): certified after the band extension */
   HPCTOPK_ROUTE_RECOVERY = 4, /* still underfilled (or view unusable): full-radix exact recovery */
-  HPCTOPK_ROUTE_OVERFLOW = 5  /* admitted tail larger than the on-chip capacity: exact recovery */
+  HPCTOPK_ROUTE_OVERFLOW = 5, /* admitted tail larger than the on-chip capacity: exact recovery */
+  HPCTOPK_ROUTE_BAND2 = 6     /* C(tau_1) < K <= C(tau_2): certified by a second, wider nested band
+                                 (sample rank ceil(3K/s)) instead of the full recovery; counted in
+                                 hpctopk_stats.rows_band2, not in rows_by_route */
 };
 
 /* Counters of the most recent hpctopk_select call on a workspace (host struct). */
@@ -62,14 +65,16 @@ typedef struct {
   uint64_t cycles_finish;     /* ... certification branch, band/recovery, Phase 3, output commit */
   uint64_t cycles_total;      /* ... whole tasks, from claim to completion */
   uint64_t cycles_detail[8];  /* finer split of the above, for tuning runs (meaning may change) */
-  uint64_t reserved[2];
+  uint64_t general_refinements; /* rows whose row-adaptive digit failed and took the 11+11+10 refinement */
+  uint64_t rows_band2;          /* rows resolved by HPCTOPK_ROUTE_BAND2 */
 } hpctopk_stats;
 
 /* Per-row record of the most recent call (host struct; see hpctopk_read_row_info). */
 typedef struct {
   int32_t route;    /* HPCTOPK_ROUTE_* */
   int32_t tau;      /* tau_0 | (tau_1 << 16) for sampled rows, -1 otherwise (Eq. "primary-threshold") */
-  int32_t c_tau0;   /* C(tau_0), Eq. "candidate-set"; L on the direct route */
+  int32_t c_tau0;   /* C(tau_0), Eq. "candidate-set"; L on the direct route; on the overflow route a
+                       lower bound (counted over the stored part of the admitted tail) */
   int32_t c_final;  /* size of the admitted tail that entered refinement (0 on recovery/short) */
 } hpctopk_row_info;
 

@@ -24,7 +24,7 @@ class Stats(ctypes.Structure):
                 ("error_flags", ctypes.c_uint64), ("cycles_phase1", ctypes.c_uint64),
                 ("cycles_scan", ctypes.c_uint64), ("cycles_finish", ctypes.c_uint64),
                 ("cycles_total", ctypes.c_uint64), ("cycles_detail", ctypes.c_uint64 * 8),
-                ("reserved", ctypes.c_uint64 * 2)]
+                ("general_refinements", ctypes.c_uint64), ("rows_band2", ctypes.c_uint64)]
 
     def as_dict(self):
         d = {f"rows_{n}": int(self.rows_by_route[i]) for i, n in enumerate(ROUTE_NAMES)}
@@ -33,7 +33,8 @@ class Stats(ctypes.Structure):
                      "cycles_finish", "cycles_total"):
             d[name] = int(getattr(self, name))
         d["cycles_detail"] = [int(v) for v in self.cycles_detail]
-        d["reserved"] = [int(v) for v in self.reserved]
+        d["general_refinements"] = int(self.general_refinements)
+        d["rows_band2"] = int(self.rows_band2)
         return d
 
 

@@ -27,8 +27,22 @@
 #ifndef HPCTOPK_EXPERIMENT
 #define HPCTOPK_EXPERIMENT 0
 #endif
+// Per-phase cycle counters (hpctopk_stats::cycles_*) are a tuning aid: reading the SM clock
+// pins the instruction schedule around it and costs measurable throughput, so the counters
+// are compiled in only with -DHPCTOPK_TIMERS=1 and read as zero otherwise.
+#ifndef HPCTOPK_TIMERS
+#define HPCTOPK_TIMERS 0
+#endif
 
 namespace {
+
+__device__ __forceinline__ long long tick() {
+#if HPCTOPK_TIMERS
+  return clock64();
+#else
+  return 0;
+#endif
+}
 
 constexpr int kBins = 2048;            // B_c and the widest refinement digit
 constexpr int kSplitRowsMax = 512;     // rows beyond this are never split (enough row parallelism)
@@ -39,8 +53,8 @@ constexpr int kSmallMax = kBins / 2;   // boundary group resolved by direct rank
 // workspace layout (bytes)
 constexpr size_t kOffCtrl = 0;                       // uint32 task_counter
 constexpr size_t kOffStats = 256;                    // hpctopk_stats (176 B)
-constexpr size_t kOffSplit = 512;                    // arrive[512], count[512]
-constexpr size_t kZeroBytes = kOffSplit + 2 * kSplitRowsMax * sizeof(uint32_t);
+constexpr size_t kOffSplit = 512;                    // arrive[512], count[512], count of A(tau_0)[512]
+constexpr size_t kZeroBytes = kOffSplit + 3 * kSplitRowsMax * sizeof(uint32_t);
 constexpr size_t kOffRowInfo = 8192;
 constexpr int kPrefetchAheadBytes = 65536;   // L2 prefetch distance inside a row's scan
 constexpr int kPrefetchHeadBytes = 131072;   // bytes of the next task's range warmed in L2 ahead of time
@@ -50,7 +64,13 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // Candidate capacity: `capacity_for` entries in total, the first `smem_capacity_for` of them in
 // shared memory and the rest in the CTA's global overflow slice (Section 5.3).
 __host__ __device__ inline int capacity_for(int K) { return 4 * K > 4096 ? 4 * K : 4096; }
+#ifndef HPCTOPK_CAPS3
 __host__ __device__ inline int smem_capacity_for(int K) { return 2 * K > 2048 ? 2 * K : 2048; }
+#else
+// 3K entries up to K = 2048 (the nested tail A(tau_1) holds about 1.75K, rarely more than 2.5K),
+// 2K above, where three CTAs of 3K entries would no longer fit one SM.
+__host__ __device__ inline int smem_capacity_for(int K) { return K <= 2048 ? (3 * K > 3072 ? 3 * K : 3072) : 2 * K; }
+#endif
 __host__ __device__ inline int stride_for(int K) {
   int s = 1;
   while (s * 2 <= 128 && s * 2 * 16 <= K) s *= 2;
@@ -74,15 +94,18 @@ struct Params {
 };
 
 struct Shared {
+  hpctopk_stats acc;         // this CTA's counters (first member of every kernel's shared state)
   uint32_t hist[kBins];
   uint32_t warp_sums[32];
   uint32_t cand_count;
   uint32_t out_count;
   uint32_t small_count;
+  uint32_t count0;           // split rows: admitted scores that also pass the tau_0 cutoff
+  uint32_t count0_cut;
   int32_t loc_bin[2];
   uint32_t loc_below[2];
   uint32_t loc_at[2];
-  uint32_t cutd[3];          // cutoffs of tau_0, tau_1 and of the bracket bin tau_hi
+  uint32_t cutd[4];          // cutoffs of tau_0, tau_1, of the bracket bin tau_hi, and of tau_2
   int32_t task;
   int32_t claim;
   uint32_t bcast0;
@@ -147,7 +170,11 @@ __global__ void init_cut_table_kernel() {
   }
 }
 
-#define DSTAMP(k, t_prev) do { if (threadIdx.x == 0) { const long long t_now = clock64(); atomicAdd(&SH().detail[k], (unsigned long long)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+#if !HPCTOPK_TIMERS
+#define DSTAMP(k, t_prev) do { (void)(t_prev); } while (0)
+#else
+#define DSTAMP(k, t_prev) do { if (threadIdx.x == 0) { const long long t_now = tick(); atomicAdd(reinterpret_cast<unsigned long long*>(&stats_of(nullptr)->cycles_detail[k]), (unsigned long long)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+#endif
 
 // ---------------------------------------------------------------- warp-level primitives
 // min{b : H(b) >= quota} over the 2048-bin histogram, by one warp: lane sums of 64 bins, warp
@@ -195,40 +222,45 @@ __device__ __forceinline__ int w_locate(const uint32_t* hist, const LaneSums ls,
   at = __shfl_sync(0xFFFFFFFFu, at_m, M);
   return __shfl_sync(0xFFFFFFFFu, bin_m, M);
 }
-// Three quotas located together: the three dependent chains of shuffles and loads advance in
+// Several quotas located together: the three dependent chains of shuffles and loads advance in
 // lockstep, so their latencies overlap instead of adding up (a warp issues in order).
-__device__ __forceinline__ void w_locate3(const uint32_t* hist, const LaneSums ls, const uint32_t (&quota)[3], int lane,
-                                          int (&bin)[3]) {
+template <int N>
+__device__ __forceinline__ void w_locate_n(const uint32_t* hist, const LaneSums ls, const uint32_t (&quota)[N], int lane,
+                                           int (&bin)[N]) {
   const uint32_t excl = ls.incl - ls.sum;
-  uint32_t hit[3];
+  uint32_t hit[N];
 #pragma unroll
-  for (int k = 0; k < 3; ++k) hit[k] = __ballot_sync(0xFFFFFFFFu, excl < quota[k] && quota[k] <= ls.incl);
-  int L[3];
-  uint32_t base[3];
-  uint2 pr[3];
+  for (int k = 0; k < N; ++k) hit[k] = __ballot_sync(0xFFFFFFFFu, excl < quota[k] && quota[k] <= ls.incl);
+  int L[N];
+  uint32_t base[N];
+  uint2 pr[N];
 #pragma unroll
-  for (int k = 0; k < 3; ++k) { L[k] = hit[k] ? __ffs(hit[k]) - 1 : 0; base[k] = __shfl_sync(0xFFFFFFFFu, excl, L[k]); }
+  for (int k = 0; k < N; ++k) { L[k] = hit[k] ? __ffs(hit[k]) - 1 : 0; base[k] = __shfl_sync(0xFFFFFFFFu, excl, L[k]); }
 #pragma unroll
-  for (int k = 0; k < 3; ++k) pr[k] = *reinterpret_cast<const uint2*>(hist + L[k] * 64 + 2 * lane);
-  uint32_t s2[3], incl2[3];
+  for (int k = 0; k < N; ++k) pr[k] = *reinterpret_cast<const uint2*>(hist + L[k] * 64 + 2 * lane);
+  uint32_t s2[N], incl2[N];
 #pragma unroll
-  for (int k = 0; k < 3; ++k) { s2[k] = pr[k].x + pr[k].y; incl2[k] = s2[k]; }
+  for (int k = 0; k < N; ++k) { s2[k] = pr[k].x + pr[k].y; incl2[k] = s2[k]; }
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
-    uint32_t n[3];
+    uint32_t n[N];
 #pragma unroll
-    for (int k = 0; k < 3; ++k) n[k] = __shfl_up_sync(0xFFFFFFFFu, incl2[k], d);
+    for (int k = 0; k < N; ++k) n[k] = __shfl_up_sync(0xFFFFFFFFu, incl2[k], d);
 #pragma unroll
-    for (int k = 0; k < 3; ++k) if (lane >= d) incl2[k] += n[k];
+    for (int k = 0; k < N; ++k) if (lane >= d) incl2[k] += n[k];
   }
 #pragma unroll
-  for (int k = 0; k < 3; ++k) {
+  for (int k = 0; k < N; ++k) {
     const uint32_t excl2 = base[k] + incl2[k] - s2[k];
     const uint32_t hit2 = __ballot_sync(0xFFFFFFFFu, excl2 < quota[k] && quota[k] <= excl2 + s2[k]);
     const int M = hit2 ? __ffs(hit2) - 1 : 0;
     const int bin_m = L[k] * 64 + 2 * lane + ((excl2 + pr[k].x >= quota[k]) ? 0 : 1);
     bin[k] = (hit[k] && hit2) ? __shfl_sync(0xFFFFFFFFu, bin_m, M) : -1;
   }
+}
+__device__ __forceinline__ void w_locate3(const uint32_t* hist, const LaneSums ls, const uint32_t (&quota)[3], int lane,
+                                          int (&bin)[3]) {
+  w_locate_n<3>(hist, ls, quota, lane, bin);
 }
 __device__ __forceinline__ void w_clear_hist(uint32_t* hist, int lane) {
   uint4* hv = reinterpret_cast<uint4*>(hist);
@@ -345,9 +377,21 @@ __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v
 // Append one admitted score: reserve a slot, store (kd, idx).  Entries beyond the capacity are
 // counted, not stored.  (The histogram of the refinement digit is built from the compacted
 // on-chip tail right after the pass, see select_adaptive; no second row pass is involved.)
+#if HPCTOPK_EXPERIMENT == 7
+constexpr bool kCount0InScan = true;
+#else
+constexpr bool kCount0InScan = false;   // C(tau_0) is counted from the stored tail after the pass
+#endif
+#ifdef HPCTOPK_WARP_APPEND
+constexpr bool kWarpAppend = true;    // experiment: warp-synchronous slot reservation (measured slower)
+#else
+constexpr bool kWarpAppend = false;
+#endif
+template <bool COUNT0>
 __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const CandCtx& c) {
   Shared& sh = SH();
   const uint32_t kd = kd_of_bits(u);
+  if (COUNT0 && kd <= sh.count0_cut) atomicAdd(&sh.count0, 1u);
 #if HPCTOPK_EXPERIMENT == 2
   const uint32_t pos = idx & 2047u; sh.cand_count = 3000;
 #else
@@ -363,7 +407,7 @@ __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const
 //   BAND = true : admit cut_lo < kd <= cut_hi.   (the band of Eq. "rescue-band")
 // Admitted scores are rare (about 1.5 K / L of the row), so the loop spends one compare and one
 // branch per score and leaves everything else to the taken branch.
-template <int THREADS, int U, bool BAND>
+template <int THREADS, int U, bool BAND, bool COUNT0 = false>
 __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
                                         uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
   const int tid = threadIdx.x;
@@ -384,7 +428,7 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
     else if (tid >= 8 && tid - 8 < ntail) e = e1 - ntail + (tid - 8);
     if (e >= 0) {
       const uint32_t u = __float_as_uint(__ldg(scores + e));
-      if (admit(u)) append_candidate(u, (uint32_t)(e - g0), cc);
+      if (admit(u)) append_candidate<COUNT0>(u, (uint32_t)(e - g0), cc);
     }
   }
   const int64_t nvec = (b1 - b0) >> 2;
@@ -397,10 +441,10 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
   auto classify = [&](const float4& f, uint32_t i) {
     const uint32_t u0 = __float_as_uint(f.x), u1 = __float_as_uint(f.y);
     const uint32_t u2 = __float_as_uint(f.z), u3 = __float_as_uint(f.w);
-    if (admit(u0)) append_candidate(u0, i + 0, cc);
-    if (admit(u1)) append_candidate(u1, i + 1, cc);
-    if (admit(u2)) append_candidate(u2, i + 2, cc);
-    if (admit(u3)) append_candidate(u3, i + 3, cc);
+    if (admit(u0)) append_candidate<COUNT0>(u0, i + 0, cc);
+    if (admit(u1)) append_candidate<COUNT0>(u1, i + 1, cc);
+    if (admit(u2)) append_candidate<COUNT0>(u2, i + 2, cc);
+    if (admit(u3)) append_candidate<COUNT0>(u3, i + 3, cc);
   };
   // The loads are fed from L2: each thread asks for the lines kPrefetchAheadBytes further on,
   // so DRAM latency is covered by requests that hold no registers.
@@ -418,9 +462,53 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
 #endif
     }
   };
+  // Whole tiles are classified warp-synchronously: every lane counts its admitted scores, one
+  // shuffle scan turns the counts into slot offsets, and one lane reserves the warp's slots with
+  // a single atomic.  (One atomic per admitted score, each waited for by a diverged lane, made
+  // the latency of the taken branch the largest term of the pass.)
+  const int lane = tid & 31;
   auto process_tile = [&](const float4 (&buf)[U], uint32_t ibase) {
+    if (COUNT0 || !kWarpAppend) {
 #pragma unroll
-    for (int j = 0; j < U; ++j) classify(buf[j], ibase + (uint32_t)(j * THREADS * 4));
+      for (int j = 0; j < U; ++j) classify(buf[j], ibase + (uint32_t)(j * THREADS * 4));
+      return;
+    }
+    uint32_t n = 0;
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      n += admit(__float_as_uint(buf[j].x)) ? 1u : 0u;
+      n += admit(__float_as_uint(buf[j].y)) ? 1u : 0u;
+      n += admit(__float_as_uint(buf[j].z)) ? 1u : 0u;
+      n += admit(__float_as_uint(buf[j].w)) ? 1u : 0u;
+    }
+    if (!__any_sync(0xFFFFFFFFu, n != 0u)) return;
+    uint32_t incl = n;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= d) incl += up;
+    }
+    uint32_t base = 0;
+    if (lane == 31) base = atomicAdd(&SH().cand_count, incl);
+    base = __shfl_sync(0xFFFFFFFFu, base, 31);
+    if (n == 0u) return;
+    uint32_t pos = base + incl - n;
+    auto put = [&](uint32_t u, uint32_t idx) {
+      if (admit(u)) {
+        const uint2 e = make_uint2(kd_of_bits(u), idx);
+        if (pos < cc.cap_s) CAND()[pos] = e;
+        else if (pos < cc.cap) cc.spill[pos - cc.cap_s] = e;
+        ++pos;
+      }
+    };
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const uint32_t i = ibase + (uint32_t)(j * THREADS * 4);
+      put(__float_as_uint(buf[j].x), i + 0);
+      put(__float_as_uint(buf[j].y), i + 1);
+      put(__float_as_uint(buf[j].z), i + 2);
+      put(__float_as_uint(buf[j].w), i + 3);
+    }
   };
 
   // Two register tiles: the loads of one are in flight while the other is classified.
@@ -450,13 +538,14 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
 struct CandidateSource {          // the admitted tail: shared memory, then the overflow slice
   CandCtx cc;
   uint32_t n;
+  uint32_t kd_max = 0xFFFFFFFFu;  // entries with a larger key are skipped (split rows hold A(tau_1))
   template <int THREADS, typename F>
   __device__ __forceinline__ void for_each(F f) const {
     for (uint32_t b = 0; b < n; b += THREADS) {
       const uint32_t i = b + threadIdx.x;
       const bool v = i < n;
       const uint2 c = v ? cand_load(cc, i) : make_uint2(0u, 0u);
-      f(v, c.x, c.y);
+      f(v && c.x <= kd_max, c.x, c.y);
     }
   }
 };
@@ -467,26 +556,31 @@ struct RowSource {                // the complete row in global memory (recovery
   template <int THREADS, typename F>
   __device__ __forceinline__ void for_each(F f) const {
     const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
-    for (int64_t base = va; base < vb; base += THREADS) {
-      const int64_t v = base + threadIdx.x;
-      const int64_t e = v << 2;
-      const bool in = v < vb;
-      const bool full = in && e >= g0 && e + 4 <= g1;
-      float x[4] = {0.f, 0.f, 0.f, 0.f};
-      bool ok[4] = {false, false, false, false};
-      if (full) {
-        const float4 t = __ldg(reinterpret_cast<const float4*>(scores + e));
-        x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
-        ok[0] = ok[1] = ok[2] = ok[3] = true;
-      } else if (in) {
+    constexpr int R = 1;       // vectors per thread in flight; 2 spills under the 40-register budget and measured slower
+    for (int64_t base = va + threadIdx.x; base < vb + threadIdx.x; base += R * THREADS) {
+      float4 x[R];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          ok[j] = (e + j >= g0) && (e + j < g1);
-          if (ok[j]) x[j] = __ldg(scores + e + j);
-        }
+      for (int k = 0; k < R; ++k) {
+        const int64_t e = (base + k * THREADS) << 2;
+        const bool full = e >= g0 && e + 4 <= g1;
+        x[k] = full ? __ldg(reinterpret_cast<const float4*>(scores + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) f(ok[j], kd_of_bits(__float_as_uint(x[j])), (uint32_t)(e + j - g0));
+      for (int k = 0; k < R; ++k) {
+        const int64_t e = (base + k * THREADS) << 2;
+        const bool full = e >= g0 && e + 4 <= g1;
+        float xs[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
+        bool ok[4] = {full, full, full, full};
+        if (!full && e < g1) {                                       // a ragged first or last vector
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            ok[j] = (e + j >= g0) && (e + j < g1);
+            if (ok[j]) xs[j] = __ldg(scores + e + j);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) f(ok[j], kd_of_bits(__float_as_uint(xs[j])), (uint32_t)(e + j - g0));
+      }
     }
   }
 };
@@ -560,24 +654,44 @@ __device__ __noinline__ void select_and_emit(const Source src, uint32_t K, bool 
 }
 
 // ---------------------------------------------------------------- per-row bookkeeping
-__device__ __forceinline__ hpctopk_stats* stats_of(unsigned char* ws) {
-  return reinterpret_cast<hpctopk_stats*>(ws + kOffStats);
+// Counters are accumulated per CTA in shared memory (the first bytes of the dynamic shared
+// segment) and added to the workspace once, when the CTA leaves: per-row global atomics on a
+// handful of addresses were a measurable serial cost.
+__device__ __forceinline__ hpctopk_stats* stats_of(unsigned char*) {
+  return reinterpret_cast<hpctopk_stats*>(smem_raw);
 }
-#define TSTAMP(P, k, t_prev) do { if (threadIdx.x == 0) { const long long t_now = clock64(); add64(&stats_of((P).ws)->cycles_detail[k], (uint64_t)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
-__device__ __forceinline__ void add64(uint64_t* p, uint64_t v);
-__device__ __forceinline__ hpctopk_stats* stats_of(unsigned char* ws);
+__device__ __forceinline__ void stats_clear() {
+  unsigned long long* a = reinterpret_cast<unsigned long long*>(smem_raw);
+  for (int i = threadIdx.x; i < (int)(sizeof(hpctopk_stats) / 8); i += blockDim.x) a[i] = 0ull;
+}
+// One thread, after every contributor of the CTA is done.
+__device__ __forceinline__ void stats_flush(unsigned char* ws) {
+  const unsigned long long* a = reinterpret_cast<const unsigned long long*>(smem_raw);
+  unsigned long long* g = reinterpret_cast<unsigned long long*>(ws + kOffStats);
+  constexpr int kMaxIdx = (int)(offsetof(hpctopk_stats, candidates_max) / 8);
+  for (int i = 0; i < (int)(sizeof(hpctopk_stats) / 8); ++i) {
+    const unsigned long long v = a[i];
+    if (v == 0ull) continue;
+    if (i == kMaxIdx) atomicMax(&g[i], v); else atomicAdd(&g[i], v);
+  }
+}
 __device__ __forceinline__ void add64(uint64_t* p, uint64_t v) {
+#if HPCTOPK_EXPERIMENT != 4
   atomicAdd(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
+#endif
 }
 __device__ __forceinline__ void max64(uint64_t* p, uint64_t v) {
+#if HPCTOPK_EXPERIMENT != 4
   atomicMax(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
+#endif
 }
 __device__ void record_row(const Params& P, int row, int route, int tau, uint32_t c0, uint32_t cfin,
                            uint64_t scanned, uint64_t sampled, uint64_t L) {
   if (threadIdx.x != 0) return;
   hpctopk_stats* st = stats_of(P.ws);
-  add64(&st->rows_by_route[route], 1);
-  if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND) {
+  if (route == HPCTOPK_ROUTE_BAND2) add64(&st->rows_band2, 1);
+  else add64(&st->rows_by_route[route], 1);
+  if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND || route == HPCTOPK_ROUTE_BAND2) {
     add64(&st->candidates_sum, cfin);
     max64(&st->candidates_max, cfin);
   }
@@ -601,7 +715,7 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   const int64_t n_view = L > a ? ((L - a + s - 1) >> bits) : 0;
   tau_pack = -1;
   if (n_view < P.q1) return false;
-  long long ts = clock64();
+  long long ts = tick();
   __syncthreads();
   clear_hist<THREADS>(sh);
   __syncthreads();
@@ -628,11 +742,13 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
     uint32_t below, at;
     int q_hi = (P.K + 2 * s - 1) / (2 * s);
     if (q_hi < 1) q_hi = 1;
-    const uint32_t quota[3] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi};
-    int tau[3];
-    w_locate3(sh.hist, ls, quota, lane, tau);
+    const uint32_t q2 = (uint32_t)((3 * P.K + s - 1) / s);             // second band: sample rank ceil(3K/s)
+    const uint32_t quota[4] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi, q2};
+    int tau[4];
+    w_locate_n<4>(sh.hist, ls, quota, lane, tau);
     (void)below; (void)at;
-    if (lane < 3) sh.cutd[lane] = g_cut_table[lane == 0 ? tau[0] : (lane == 1 ? tau[1] : tau[2])];
+    if (tau[3] < 0) tau[3] = tau[1];                                  // view shorter than q2: no second band
+    if (lane < 4) sh.cutd[lane] = g_cut_table[lane == 0 ? tau[0] : (lane == 1 ? tau[1] : (lane == 2 ? tau[2] : tau[3]))];
     if (lane == 0) { sh.loc_bin[0] = tau[0]; sh.loc_bin[1] = tau[1]; }
   }
   __syncthreads();
@@ -662,7 +778,7 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
     const uint32_t d = (cut_base - kd) >> shv;
     return 2047u - (d < 2047u ? d : 2047u);
   };
-  long long ts = clock64();
+  long long ts = tick();
   __syncthreads();
   clear_hist<THREADS>(sh);
   if (tid == 0) { sh.out_count = 0; sh.small_count = 0; }
@@ -672,7 +788,11 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
     uint2 c[4];
     bool v[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) { const uint32_t i = i0 + k * THREADS + tid; v[k] = i < C; c[k] = v[k] ? cand_load(cc, i) : make_uint2(0u, 0u); }
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t i = i0 + k * THREADS + tid;
+      c[k] = i < C ? cand_load(cc, i) : make_uint2(0xFFFFFFFFu, 0u);
+      v[k] = i < C && c[k].x <= cut_base;       // a split row's buffer also holds the band beyond tau_0
+    }
 #pragma unroll
     for (int k = 0; k < 4; ++k) if (v[k]) atomicAdd(&sh.hist[digit(c[k].x)], 1u);
   }
@@ -699,8 +819,8 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const uint32_t i = i0 + k * THREADS + tid;
-      c[k] = i < C ? cand_load(cc, i) : make_uint2(0u, 0u);
-      dg[k] = i < C ? digit(c[k].x) : 0xFFFFFFFFu;
+      c[k] = i < C ? cand_load(cc, i) : make_uint2(0xFFFFFFFFu, 0u);
+      dg[k] = (i < C && c[k].x <= cut_base) ? digit(c[k].x) : 0xFFFFFFFFu;
       cnt += dg[k] < (uint32_t)b ? 1u : 0u;
     }
     const uint32_t incl = warp_inclusive_scan<THREADS>(cnt);
@@ -751,44 +871,57 @@ __device__ void emit_short_row(const Params& P, int row, int64_t g0, int64_t L) 
   }
 }
 
-// Everything after the primary pass of a sampled row: certification branch (Section 4.3),
-// band extension, refinement or exact recovery, output commit.  On entry the shared candidate
-// arrays hold min(C0, cap) entries of A(tau_0) and sh.hist their leading-digit histogram iff
-// `hist_ready`.
+// C(tau_0) of the stored part of the nested tail: entries whose key passes the tau_0 cutoff.
+// Adds into sh.count0 (cleared by the caller before the pass).
+template <int THREADS>
+__device__ __forceinline__ void count_primary(const CandCtx& cc, uint32_t n, uint32_t cut0) {
+  Shared& sh = SH();
+  uint32_t c = 0;
+  for (uint32_t i = threadIdx.x; i < n; i += THREADS) c += cand_load(cc, i).x <= cut0 ? 1u : 0u;
+  c = __reduce_add_sync(0xFFFFFFFFu, c);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(&sh.count0, c);
+  __syncthreads();
+}
+
+// Everything after the complete-row pass of a sampled row: certification branch (Section 4.3),
+// refinement or exact recovery, output commit.  The pass admitted the nested tail A(tau_1) and
+// counted A(tau_0) inside it, so the band extension of an underfilled primary boundary costs no
+// second pass: C(tau_0) >= K refines the entries with kd <= cut(tau_0), C(tau_0) < K <= C(tau_1)
+// all of them.  A row that is still underfilled appends one wider band (tau_1, tau_2] in a
+// second pass before it falls back to the storage-free recovery.  On entry the candidate arrays
+// hold min(C1, cap) entries and sh.cand_count == C1.
 template <int THREADS, int U>
-__device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t L, uint32_t C0,
-                                   bool hist_ready, int tau_pack, uint64_t scanned, uint64_t sampled) {
+__device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t L, uint32_t C0, uint32_t C1,
+                                   int tau_pack, uint64_t scanned, uint64_t sampled) {
   Shared& sh = SH();
   const CandCtx cc = cand_ctx(P);
   int32_t* oi = P.out_idx + (int64_t)row * P.K;
   float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
   const uint32_t K = (uint32_t)P.K, cap = (uint32_t)P.cap;
   int route;
-  uint32_t cfin = 0;
-  if (C0 > cap) {
+  uint32_t cfin = 0, C = C1, cut_base = 0;
+  if (C1 > cap) {
     route = HPCTOPK_ROUTE_OVERFLOW;
   } else if (C0 >= K) {
-    route = HPCTOPK_ROUTE_PRIMARY;
-    cfin = C0;
+    route = HPCTOPK_ROUTE_PRIMARY; cfin = C0; cut_base = sh.cutd[0];
+  } else if (C1 >= K) {
+    route = HPCTOPK_ROUTE_BAND; cfin = C1; cut_base = sh.cutd[1];
   } else {
-    // band extension: append tau_0 < c(x) <= tau_1 and extend the histogram (Eq. "rescue-hist")
-    __syncthreads();
-    scan_range<THREADS, U, true>(P.scores, g0, g0, g0 + L, sh.cutd[0], sh.cutd[1], cc);
-    __syncthreads();
-    scanned += (uint64_t)L;
-    const uint32_t C1 = sh.cand_count;
-    if (C1 > cap) route = HPCTOPK_ROUTE_OVERFLOW;
-    else if (C1 >= K) { route = HPCTOPK_ROUTE_BAND; cfin = C1; }
-    else route = HPCTOPK_ROUTE_RECOVERY;
+    route = HPCTOPK_ROUTE_RECOVERY;
+    if (sh.cutd[3] > sh.cutd[1]) {
+      __syncthreads();
+      scan_range<THREADS, U, true>(P.scores, g0, g0, g0 + L, sh.cutd[1], sh.cutd[3], cc);
+      __syncthreads();
+      scanned += (uint64_t)L;
+      const uint32_t C2 = sh.cand_count;
+      if (C2 >= K && C2 <= cap) { route = HPCTOPK_ROUTE_BAND2; cfin = C2; C = C2; cut_base = sh.cutd[3]; }
+    }
   }
-  if (route == HPCTOPK_ROUTE_PRIMARY || route == HPCTOPK_ROUTE_BAND) {
-    const uint32_t cut_base = route == HPCTOPK_ROUTE_BAND ? sh.cutd[1] : sh.cutd[0];
-    if (!select_adaptive<THREADS>(cc, cfin, K, cut_base, sh.cutd[2], oi, ov)) {
-      if (threadIdx.x == 0) add64(&stats_of(P.ws)->reserved[0], 1);      // general refinement taken
+  if (cfin) {
+    if (!select_adaptive<THREADS>(cc, C, K, cut_base, sh.cutd[2], oi, ov)) {
+      if (threadIdx.x == 0) add64(&stats_of(P.ws)->general_refinements, 1);
       __syncthreads();
-      clear_hist<THREADS>(sh);
-      __syncthreads();
-      CandidateSource cs{cc, cfin};
+      CandidateSource cs{cc, C, cut_base};
       select_and_emit<THREADS>(cs, K, false, oi, ov);
     }
   } else {
@@ -829,28 +962,27 @@ __device__ void process_row(const Params& P, int row) {
     return;
   }
   int tau_pack;
-  const long long t0 = clock64();
+  const long long t0 = tick();
   if (!phase1<THREADS>(P, row, g0, L, tau_pack)) {
     RowSource rs{P.scores, g0, g0 + L};
     select_and_emit<THREADS>(rs, K, false, oi, ov);
     record_row(P, row, HPCTOPK_ROUTE_RECOVERY, -1, 0, 0, 4ull * (uint64_t)L, 0, (uint64_t)L);
     return;
   }
-  const long long t1 = clock64();
+  const long long t1 = tick();
   const uint64_t sampled = (uint64_t)((L + P.stride - 1) / P.stride);
-  clear_hist<THREADS>(sh);
-  if (threadIdx.x == 0) sh.cand_count = 0;
+  if (threadIdx.x == 0) { sh.cand_count = 0; sh.count0 = 0; sh.count0_cut = sh.cutd[0]; }
   __syncthreads();
-  scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[0], cc);
+  scan_range<THREADS, U, false, kCount0InScan>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[1], cc);
   __syncthreads();
-  const long long t2 = clock64();
-  const uint32_t C0 = sh.cand_count;
-  finish_sampled_row<THREADS, U>(P, row, g0, L, C0, true, tau_pack, (uint64_t)L, sampled);
+  if (!kCount0InScan) count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
+  const long long t2 = tick();
+  finish_sampled_row<THREADS, U>(P, row, g0, L, sh.count0, sh.cand_count, tau_pack, (uint64_t)L, sampled);
   if (threadIdx.x == 0) {
     hpctopk_stats* st = stats_of(P.ws);
     add64(&st->cycles_phase1, (uint64_t)(t1 - t0));
     add64(&st->cycles_scan, (uint64_t)(t2 - t1));
-    add64(&st->cycles_finish, (uint64_t)(clock64() - t2));
+    add64(&st->cycles_finish, (uint64_t)(tick() - t2));
   }
 }
 
@@ -870,9 +1002,9 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   uint2* gcand = reinterpret_cast<uint2*>(P.ws + cand_off) + (size_t)row * cap;
 
   int tau_pack;
-  const long long t0 = clock64();
+  const long long t0 = tick();
   const bool usable = phase1<THREADS>(P, row, g0, L, tau_pack);
-  const long long t1 = clock64();
+  const long long t1 = tick();
   const uint64_t sampled = usable ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
   // contiguous, 16-byte aligned partition of the row's vectors
   const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
@@ -881,16 +1013,20 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   if (e0 < g0) e0 = g0;
   if (e1 > g1) e1 = g1;
   if (e1 < e0) e1 = e0;
+  // A split row admits the nested tail A(tau_1) in its one pass (and counts A(tau_0) inside it),
+  // so that an underfilled primary boundary never costs the finisher a second, single-CTA pass.
+  uint32_t* rowcnt0 = rowcnt + kSplitRowsMax;
   __syncthreads();
-  if (threadIdx.x == 0) sh.cand_count = 0;
-  clear_hist<THREADS>(sh);
+  if (threadIdx.x == 0) { sh.cand_count = 0; sh.count0 = 0; sh.count0_cut = sh.cutd[0]; }
   __syncthreads();
-  if (usable) scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, sh.cutd[0], cc);
+  if (usable) scan_range<THREADS, U, false, kCount0InScan>(P.scores, g0, e0, e1, 0u, sh.cutd[1], cc);
   __syncthreads();
+  if (usable && !kCount0InScan) count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
   const uint32_t Cp = sh.cand_count;
-  const long long t2 = clock64();
+  const long long t2 = tick();
   if (threadIdx.x == 0) {
     sh.bcast0 = atomicAdd(&rowcnt[row], Cp);
+    atomicAdd(&rowcnt0[row], sh.count0);
     hpctopk_stats* st = stats_of(P.ws);
     add64(&st->cycles_phase1, (uint64_t)(t1 - t0));
     add64(&st->cycles_scan, (uint64_t)(t2 - t1));
@@ -909,7 +1045,8 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   if (sh.bcast1 != (uint32_t)(nseg - 1)) return;      // not the last arriver
   // ---- finisher: C(tau_0) = sum_p C_p, A(tau_0) = union of the published ranges (Eq. "split-reduce")
   __threadfence();
-  const uint32_t C0 = *reinterpret_cast<volatile uint32_t*>(&rowcnt[row]);
+  const uint32_t C1 = *reinterpret_cast<volatile uint32_t*>(&rowcnt[row]);      // C(tau_1)
+  const uint32_t C0 = *reinterpret_cast<volatile uint32_t*>(&rowcnt0[row]);     // C(tau_0)
   if (threadIdx.x == 0) add64(&stats_of(P.ws)->rows_split, 1);
   if (!usable) {
     RowSource rs{P.scores, g0, g1};
@@ -918,14 +1055,14 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
     record_row(P, row, HPCTOPK_ROUTE_RECOVERY, -1, 0, 0, 4ull * (uint64_t)L, 0, (uint64_t)L);
     return;
   }
-  if (C0 <= cap) {
-    for (uint32_t i = threadIdx.x; i < C0; i += THREADS) cand_store(cc, i, __ldcg(gcand + i));
+  __syncthreads();
+  if (C1 <= cap) {
+    for (uint32_t i = threadIdx.x; i < C1; i += THREADS) cand_store(cc, i, __ldcg(gcand + i));
   }
+  if (threadIdx.x == 0) sh.cand_count = C1;
   __syncthreads();
-  if (threadIdx.x == 0) sh.cand_count = C0;
-  __syncthreads();
-  finish_sampled_row<THREADS, U>(P, row, g0, L, C0, false, tau_pack, 0, 0);
-  if (threadIdx.x == 0) add64(&stats_of(P.ws)->cycles_finish, (uint64_t)(clock64() - t2));
+  finish_sampled_row<THREADS, U>(P, row, g0, L, C0, C1, tau_pack, 0, 0);
+  if (threadIdx.x == 0) add64(&stats_of(P.ws)->cycles_finish, (uint64_t)(tick() - t2));
 }
 
 // ---------------------------------------------------------------- the persistent kernel
@@ -955,6 +1092,16 @@ __device__ __forceinline__ void prefetch_head(const Params& P, int64_t e0, int64
     asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
 }
 
+// Unsplit calls hand rows out from the end of the batch: causal prefill lists rows by growing
+// length, so this runs the longest rows first and leaves short ones to fill the tail of the grid.
+__device__ __forceinline__ int row_of_task(const Params& P, uint32_t task) {
+#if HPCTOPK_EXPERIMENT == 6
+  return (int)task;
+#else
+  return P.num_rows - 1 - (int)task;
+#endif
+}
+
 template <int THREADS, int U, int MINB>
 __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) {
   Shared& sh = SH();
@@ -962,7 +1109,7 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
   uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl);
   const int tid = threadIdx.x;
 
-  if (tid == 0) sh.detail = reinterpret_cast<unsigned long long*>(P.ws + kOffStats + offsetof(hpctopk_stats, cycles_detail));
+  stats_clear();
   __syncthreads();
   uint32_t total_tasks = (uint32_t)P.num_rows;
   if (P.split_enabled) {
@@ -1016,11 +1163,12 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
   uint32_t task = blockIdx.x;
   uint32_t next = blockIdx.x + gridDim.x;
   while (task < total_tasks) {
-    const long long task_t0 = clock64();
+    const long long task_t0 = tick();
     if (tid == 0) sh.claim = (int32_t)(2u * gridDim.x + atomicAdd(task_counter, 1u));
     if (!P.split_enabled && next < total_tasks) {
-      prefetch_view<THREADS>(P, (int)next);
-      const int64_t ng0 = P.row_starts[next], nL = P.row_lengths[next];
+      const int nrow = row_of_task(P, next);
+      prefetch_view<THREADS>(P, nrow);
+      const int64_t ng0 = P.row_starts[nrow], nL = P.row_lengths[nrow];
       if (nL > P.K) prefetch_head<THREADS>(P, ng0, ng0 + nL);
     }
     if (P.split_enabled) {
@@ -1032,18 +1180,20 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
       if (nseg <= 1) process_row<THREADS, U>(P, row);
       else process_segment<THREADS, U>(P, row, (int)(task - seg_base[row]), nseg);
     } else {
-      process_row<THREADS, U>(P, (int)task);
+      process_row<THREADS, U>(P, row_of_task(P, task));
     }
     __syncthreads();
     const uint32_t claimed = (uint32_t)sh.claim;
     if (tid == 0) {
       add64(&stats_of(P.ws)->tasks, 1);
-      add64(&stats_of(P.ws)->cycles_total, (uint64_t)(clock64() - task_t0));
+      add64(&stats_of(P.ws)->cycles_total, (uint64_t)(tick() - task_t0));
     }
     __syncthreads();
     task = next;
     next = claimed;
   }
+  __syncthreads();
+  if (tid == 0) stats_flush(P.ws);
 }
 
 }  // namespace
@@ -1051,8 +1201,14 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
 #define HPCTOPK_WS_NAMESPACE wsf     // namespace wsf: single-role variant, warp-synchronous compaction
 #define HPCTOPK_WS_FUSED 1
 #define HPCTOPK_NS 16
-#define HPCTOPK_WS_U 2
-#define HPCTOPK_WS_MINB 2
+#ifndef HPCTOPK_FUSED_MINB
+#define HPCTOPK_FUSED_MINB 2
+#endif
+#ifndef HPCTOPK_FUSED_U
+#define HPCTOPK_FUSED_U 2
+#endif
+#define HPCTOPK_WS_U HPCTOPK_FUSED_U
+#define HPCTOPK_WS_MINB HPCTOPK_FUSED_MINB
 #include "hpctopk_ws.cuh"
 namespace {
 
@@ -1071,10 +1227,14 @@ const Variant kVariants[] = {
     {hpctopk_kernel<512, 2, 3>, 512},
     {hpctopk_kernel<384, 2, 4>, 384},
     {hpctopk_kernel<640, 2, 2>, 640},
+    {hpctopk_kernel<512, 1, 3>, 512},
+    {hpctopk_kernel<1024, 1, 1>, 1024},
+    {hpctopk_kernel<1024, 2, 1>, 1024},
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 // 0 selects the warp-specialised kernel, v >= 1 the single-role kernel kVariants[v - 1].
-constexpr int kDefaultVariant = 1;
+constexpr int kDefaultVariant = 4;
+constexpr int kSplitVariant = 1;
 constexpr int kFusedVariant = 100;     // single-role kernel with warp-synchronous compaction (namespace wsf)
 
 struct DeviceInfo {
@@ -1089,6 +1249,13 @@ size_t smem_bytes_for(int cap_s, bool split) {
   size_t b = align_up(sizeof(Shared), 16) + (size_t)cap_s * 8;
   if (split) b += (kSplitRowsMax + 1) * sizeof(uint32_t);
   return align_up(b, 16);
+}
+
+// Index into kVariants for a call: calls with few rows (split mode) are latency-bound and
+// prefer fewer, fatter CTAs per SM than the streaming default.
+int variant_index(int variant, bool split) {
+  const int v = (variant == kDefaultVariant && split) ? kSplitVariant : variant;
+  return (v > 0 && v <= kNumVariants) ? v - 1 : 0;
 }
 
 // Shared memory is sized by capacity class so that occupancy (and the grid) depends on K only.
@@ -1170,13 +1337,13 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
       cudaGetLastError();
       return HPCTOPK_ERR_CUDA;
     }
-    const Variant& v = kVariants[(di.variant > 0 && di.variant <= kNumVariants) ? di.variant - 1 : 0];
     const size_t max_smem = smem_bytes_for(class_cap_s(2), true);
-    if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
-      cudaGetLastError();
-      return HPCTOPK_ERR_CUDA;
-    }
-    for (int sp = 0; sp < 2; ++sp)
+    for (int sp = 0; sp < 2; ++sp) {
+      const Variant& v = kVariants[variant_index(di.variant, sp != 0)];
+      if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
+        cudaGetLastError();
+        return HPCTOPK_ERR_CUDA;
+      }
       for (int c = 0; c < 3; ++c) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, v.fn, v.threads, smem_bytes_for(class_cap_s(c), sp != 0)) != cudaSuccess || n < 1) {
@@ -1185,9 +1352,10 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
         }
         di.ctas_per_sm[sp][c] = n;
       }
+    }
     di.ready = true;
   }
-  const Variant& v = kVariants[(di.variant > 0 && di.variant <= kNumVariants) ? di.variant - 1 : 0];
+  const Variant& v = kVariants[variant_index(di.variant, split)];
   const int cls = cap_class(K);
   Params P;
   P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;

@@ -89,8 +89,10 @@ struct Desc {
   int32_t pad;
 };
 
+static_assert(sizeof(hpctopk_stats) % 16 == 0, "counters must keep 16-byte alignment of what follows");
 static_assert(sizeof(HelperShared) % 16 == 0, "helper state must keep 16-byte alignment");
 struct WsShared {
+  hpctopk_stats acc;         // this CTA's counters (first member of every kernel's shared state)
   HelperShared h[kSlots];
   uint32_t cnt[kSlots][32];  // admitted scores per region of each slot's buffer
   Desc desc[kSlots];
@@ -99,6 +101,7 @@ struct WsShared {
   uint32_t warp_sums[32];    // prologue only
   uint32_t total_tasks;
   int32_t abort;
+  uint32_t groups_done;      // helper groups that have finished (the last one flushes the counters)
   unsigned long long* detail;
 };
 
@@ -107,7 +110,11 @@ __device__ __forceinline__ uint2* WCAND(int slot, uint32_t region_entries) {
   return reinterpret_cast<uint2*>(smem_raw + ((sizeof(WsShared) + 15) / 16 * 16)) + (size_t)slot * NS * region_entries;
 }
 
-#define WSTAMP(k, t_prev) do { if (G.tid() == 0) { const long long t_now = clock64(); atomicAdd(&WSH().detail[k], (unsigned long long)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+#if HPCTOPK_TIMERS
+#define WSTAMP(k, t_prev) do { if (G.tid() == 0) { const long long t_now = tick(); atomicAdd(&WSH().detail[k], (unsigned long long)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+#else
+#define WSTAMP(k, t_prev) do { (void)(t_prev); } while (0)
+#endif
 
 // ---------------------------------------------------------------- mbarrier helpers (bounded waits)
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -444,7 +451,7 @@ struct RowSrc {                   // the complete row in global memory (recovery
 template <typename Source>
 __device__ __noinline__ void g_select_and_emit(const Grp G, const Source src, uint32_t K, int32_t* out_idx, float* out_val) {
   HelperShared& sh = WSH().h[G.g];
-  long long ts = clock64();
+  long long ts = tick();
   const int shifts[6] = {53, 42, 32, 21, 10, 0};
   const int widths[6] = {11, 11, 10, 11, 11, 10};
   uint64_t prefix = 0;
@@ -525,7 +532,7 @@ __device__ __noinline__ bool g_phase1(const Grp G, const Params& P, int row, int
   const int64_t n_view = L > a ? ((L - a + s - 1) >> bits) : 0;
   tau_pack = -1;
   if (n_view < P.q1) return false;
-  long long ts = clock64();
+  long long ts = tick();
   G.sync();
   g_clear_hist(G, sh);
   G.sync();
@@ -619,7 +626,7 @@ __device__ __noinline__ Phase1Out w_phase1(const Grp G, const Params& P, int row
   const int a = bits ? (int)(__brev((uint32_t)(row & (s - 1))) >> (32 - bits)) : 0;
   const int64_t n_view = L > a ? ((L - a + s - 1) >> bits) : 0;
   if (n_view < P.q1) return o;
-  long long ts = clock64();
+  long long ts = tick();
   G.sync();
   if (wi == 0) w_clear_hist(sh.hist, lane);
   G.sync();
@@ -674,7 +681,7 @@ __device__ __noinline__ bool w_select_adaptive(const Grp G, const Buf buf, bool 
                                                uint32_t cut_hi, int32_t* out_idx, float* out_val) {
   HelperShared& sh = WSH().h[G.g];
   const int lane = G.tid() & 31, wi = G.tid() >> 5;     // lane and warp index inside the group
-  long long ts = clock64();
+  long long ts = tick();
   const uint32_t span = cut_base > cut_hi ? cut_base - cut_hi : 0u;
   int shv = 0;
   while (shv < 31 && (span >> shv) >= 2047u) ++shv;
@@ -848,11 +855,11 @@ __device__ __noinline__ void scanner_main(const Params& P, uint32_t rw, uint32_t
     for (int s = 0; s < kSlots; ++s) {
       if ((done >> s) & 1u) continue;
       int ok = 0;
-      const long long tw0 = clock64();
+      const long long tw0 = tick();
       if (lane == 0) ok = mbar_wait(&sh.posted[s], (parity >> s) & 1u) ? 1 : 0;   // one poller per warp
       ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
       if (!ok) return;
-      const long long tw1 = clock64();
+      const long long tw1 = tick();
       if (tid == 0) atomicAdd(&sh.detail[6], (unsigned long long)(tw1 - tw0));
       parity ^= 1u << s;
       const Desc d = sh.desc[s];
@@ -864,7 +871,7 @@ __device__ __noinline__ void scanner_main(const Params& P, uint32_t rw, uint32_t
       if (lane == 0) sh.cnt[s][warp] = wbase;
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.scanned[s]);
-      if (tid == 0) atomicAdd(&sh.detail[7], (unsigned long long)(clock64() - tw1));
+      if (tid == 0) atomicAdd(&sh.detail[7], (unsigned long long)(tick() - tw1));
     }
   }
 }
@@ -957,15 +964,15 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
         continue;
       }
       if (L <= (int64_t)P.cap) {                   // direct route: the whole row is admitted
-        t.e0 = g0; t.e1 = g0 + L; t.t_post = clock64();
+        t.e0 = g0; t.e1 = g0 + L; t.t_post = tick();
         post(MODE_SCAN, g0, t.e0, t.e1, 0u, 0xFFFFFFFFu);
         return true;
       }
-      const long long t0 = clock64();
+      const long long t0 = tick();
       const Phase1Out p1 = w_phase1(G, P, row, g0, L);
       const bool usable = p1.usable;
       t.tau_pack = p1.tau_pack;
-      if (ht == 0) add64(&stats_of(P.ws)->cycles_phase1, (uint64_t)(clock64() - t0));
+      if (ht == 0) add64(&stats_of(P.ws)->cycles_phase1, (uint64_t)(tick() - t0));
       t.sampled = usable ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
       if (!usable && nseg == 1) { recover_row(HPCTOPK_ROUTE_RECOVERY, 0, 0); continue; }
       int64_t e0 = g0, e1 = g0 + L;
@@ -981,7 +988,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
       t.cut0 = p1.cut0;
       t.cut1 = p1.cut1;
       t.cut_hi = p1.cut_hi;
-      t.e0 = e0; t.e1 = e1; t.t_post = clock64();
+      t.e0 = e0; t.e1 = e1; t.t_post = tick();
       t.scanned = (uint64_t)(e1 - e0);
       post(MODE_SCAN, g0, e0, e1, 0u, t.cut0);
       return true;
@@ -991,7 +998,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
   // Retires the posted task after the scanners are done with it.  Returns false when the same
   // row went back to the scanners (band extension), true when the slot is free again.
   auto complete = [&]() -> bool {
-    const long long tc0 = clock64();
+    const long long tc0 = tick();
     if (ht == 0) add64(&stats_of(P.ws)->cycles_scan, (uint64_t)(tc0 - t.t_post));
     const bool direct = t.L <= (int64_t)P.cap;
     Tally ty = buf_tally(buf);
@@ -1045,7 +1052,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
       bool done = false;
       done = w_select_adaptive(G, buf, ty.spilled, K, t.banded ? t.cut1 : t.cut0, t.cut_hi, oi, ov);
       if (!done) {
-        if (ht == 0) add64(&stats_of(P.ws)->reserved[0], 1);      // general refinement taken
+        if (ht == 0) add64(&stats_of(P.ws)->general_refinements, 1);      // general refinement taken
         BufSource bs{buf, ty.spilled};
         g_select_and_emit(G, bs, K, oi, ov);
       }
@@ -1055,13 +1062,13 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
       // band extension (Eq. "rescue-band"): same slot, same buffer, appended by the scanners
       t.banded = 1;
       t.scanned += (uint64_t)t.L;
-      t.t_post = clock64();
+      t.t_post = tick();
       post(MODE_BAND, t.g0, t.g0, t.g0 + t.L, t.cut0, t.cut1);
       return false;
     } else {
       recover_row(HPCTOPK_ROUTE_RECOVERY, t.c0, t.scanned);
     }
-    if (ht == 0) add64(&stats_of(P.ws)->cycles_finish, (uint64_t)(clock64() - tc0));
+    if (ht == 0) add64(&stats_of(P.ws)->cycles_finish, (uint64_t)(tick() - tc0));
     return true;
   };
 
@@ -1077,7 +1084,12 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
     if (complete()) busy = start_next();
   }
   post(MODE_DONE, 0, 0, 0, 0u, 0u);       // releases the scanners from this slot
-  if (ht == 0 && *reinterpret_cast<volatile int32_t*>(&wsh.abort)) add64(&stats_of(P.ws)->error_flags, 1);
+  G.sync();
+  if (ht == 0) {
+    if (*reinterpret_cast<volatile int32_t*>(&wsh.abort)) add64(&stats_of(P.ws)->error_flags, 1);
+    __threadfence_block();
+    if (atomicAdd(&wsh.groups_done, 1u) == (uint32_t)(kSlots - 1)) { __threadfence_block(); stats_flush(P.ws); }
+  }
 }
 
 template <int U>
@@ -1088,9 +1100,11 @@ __global__ void __launch_bounds__(THREADS, kMinBlocks) hpctopk_ws_kernel(const P
   const uint32_t sw = (uint32_t)ws_region_total(P.K);     // overflow entries per region (a power of two)
   uint32_t* const seg_base = reinterpret_cast<uint32_t*>(WCAND(kSlots, rw));   // after the buffers
 
+  stats_clear();
   if (tid == 0) {
     sh.detail = reinterpret_cast<unsigned long long*>(stats_of(P.ws)->cycles_detail);
     sh.abort = 0;
+    sh.groups_done = 0;
     for (int s = 0; s < kSlots; ++s) { mbar_init(&sh.posted[s], 1); mbar_init(&sh.scanned[s], NS); }
   }
   __syncthreads();

@@ -60,7 +60,8 @@ def test_config3_prefill_chunk_full_size_sampled_rows():
     srt = np.sort(got_idx, axis=1)
     assert (np.diff(srt, axis=1) > 0).all()             # K distinct indices per row
     assert stats["rows_split"] == 0
-    assert stats["rows_primary"] + stats["rows_band"] + stats["rows_recovery"] + stats["rows_overflow"] == 4096
+    assert (stats["rows_primary"] + stats["rows_band"] + stats["rows_band2"] + stats["rows_recovery"]
+            + stats["rows_overflow"]) == 4096
 
 
 @pytest.mark.parametrize("K", [2048, 4096])
