@@ -24,9 +24,6 @@
 
 #include "../../include/hpctopk.h"
 
-#ifndef HPCTOPK_EXPERIMENT
-#define HPCTOPK_EXPERIMENT 0
-#endif
 // Per-phase cycle counters (hpctopk_stats::cycles_*) are a tuning aid: reading the SM clock
 // pins the instruction schedule around it and costs measurable throughput, so the counters
 // are compiled in only with -DHPCTOPK_TIMERS=1 and read as zero otherwise.
@@ -100,11 +97,10 @@ struct Shared {
   uint32_t cand_count;
   uint32_t out_count;
   uint32_t small_count;
-  uint32_t count0;           // split rows: admitted scores that also pass the tau_0 cutoff
-  uint32_t count0_cut;
-  int32_t loc_bin[2];
-  uint32_t loc_below[2];
-  uint32_t loc_at[2];
+  uint32_t count0;           // C(tau_0) within the stored nested tail
+  int32_t loc_bin[4];
+  uint32_t loc_below[4];
+  uint32_t loc_at[4];
   uint32_t cutd[4];          // cutoffs of tau_0, tau_1, of the bracket bin tau_hi, and of tau_2
   int32_t task;
   int32_t claim;
@@ -174,6 +170,12 @@ __global__ void init_cut_table_kernel() {
 #define DSTAMP(k, t_prev) do { (void)(t_prev); } while (0)
 #else
 #define DSTAMP(k, t_prev) do { if (threadIdx.x == 0) { const long long t_now = tick(); atomicAdd(reinterpret_cast<unsigned long long*>(&stats_of(nullptr)->cycles_detail[k]), (unsigned long long)(t_now - (t_prev))); (t_prev) = t_now; } } while (0)
+#endif
+
+#if HPCTOPK_TIMERS == 2      // finer stamps inside Phase 1, in slots the refinement stamps otherwise use
+#define DSTAMP1(k, t_prev) DSTAMP(k, t_prev)
+#else
+#define DSTAMP1(k, t_prev) do { (void)(t_prev); } while (0)
 #endif
 
 // ---------------------------------------------------------------- warp-level primitives
@@ -301,12 +303,12 @@ __device__ __forceinline__ uint32_t warp_inclusive_scan(uint32_t v) {
 // Contains block barriers; every thread must call it.  Leaves sh.hist unchanged.
 template <int THREADS>
 __device__ void locate(Shared& sh, uint32_t quota0, uint32_t quota1, int nq) {
-  constexpr int BPT = kBins / THREADS;
+  constexpr int BPT = (kBins + THREADS - 1) / THREADS;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t h[BPT];
   uint32_t sum = 0;
 #pragma unroll
-  for (int b = 0; b < BPT; ++b) { h[b] = sh.hist[tid * BPT + b]; sum += h[b]; }
+  for (int b = 0; b < BPT; ++b) { h[b] = tid * BPT + b < kBins ? sh.hist[tid * BPT + b] : 0u; sum += h[b]; }
   const uint32_t incl = warp_inclusive_scan<THREADS>(sum);
   if (lane == 31) sh.warp_sums[warp] = incl;
   if (tid < 2) sh.loc_bin[tid] = -1;
@@ -324,6 +326,61 @@ __device__ void locate(Shared& sh, uint32_t quota0, uint32_t quota1, int nq) {
           sh.loc_bin[qi] = tid * BPT + b; sh.loc_below[qi] = run; sh.loc_at[qi] = h[b];
         }
         run += h[b];
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// The same for N <= 4 quotas with every warp taking part: a thread owns 4 (8 below 512 threads)
+// consecutive bins read as 16-byte vectors, so the critical path is one vector load, one warp
+// scan, one barrier and a look at the warp totals, whatever the other CTAs of the SM are doing.
+// (A single warp walking the histogram takes 13 K to 18 K cycles per row next to streaming CTAs,
+// against about 6 K here, yet the whole call ran 3 % slower with this form: the idle warps of the
+// single-warp search cost nothing, the fifteen extra warps here take issue slots from the CTAs
+// that are streaming.  Kept for tuning runs: -DHPCTOPK_P1_BLOCK, -DHPCTOPK_SA_BLOCK.)
+template <int THREADS, int N>
+__device__ __forceinline__ void locate_n(const uint32_t (&quota)[N]) {
+  Shared& sh = SH();
+  constexpr int BPT = THREADS >= 512 ? 4 : 8;
+  constexpr int NT = kBins / BPT, NW = NT / 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t h[BPT];
+  uint32_t sum = 0;
+  if (tid < NT) {
+    const uint4* hv = reinterpret_cast<const uint4*>(sh.hist) + tid * (BPT / 4);
+#pragma unroll
+    for (int v = 0; v < BPT / 4; ++v) {
+      const uint4 x = hv[v];
+      h[4 * v] = x.x; h[4 * v + 1] = x.y; h[4 * v + 2] = x.z; h[4 * v + 3] = x.w;
+      sum += x.x + x.y + x.z + x.w;
+    }
+  }
+  uint32_t incl = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= d) incl += up;
+  }
+  if (lane == 31 && warp < NW) sh.warp_sums[warp] = incl;
+  if (tid < N) sh.loc_bin[tid] = -1;
+  __syncthreads();
+  if (tid < NT) {
+    uint32_t woff = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { const uint32_t ws = sh.warp_sums[w]; woff += w < warp ? ws : 0u; }
+    const uint32_t excl = woff + incl - sum;
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+      if (excl < quota[k] && quota[k] <= excl + sum) {
+        uint32_t run = excl;
+#pragma unroll
+        for (int b = 0; b < BPT; ++b) {
+          if (run < quota[k] && run + h[b] >= quota[k]) {
+            sh.loc_bin[k] = tid * BPT + b; sh.loc_below[k] = run; sh.loc_at[k] = h[b];
+          }
+          run += h[b];
+        }
       }
     }
   }
@@ -367,7 +424,7 @@ __device__ __forceinline__ CandCtx cand_ctx(const Params& P) {
   c.spill = reinterpret_cast<uint2*>(P.ws + spill_off) + (size_t)blockIdx.x * (size_t)(P.cap - P.cap_s);
   return c;
 }
-__device__ __forceinline__ uint2 cand_load(const CandCtx& c, uint32_t i) {
+__device__ __forceinline__ uint2 cand_load(const CandCtx& c, uint32_t i) {   // (kd, idx)
   return i < c.cap_s ? CAND()[i] : __ldcg(c.spill + (i - c.cap_s));
 }
 __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v) {
@@ -377,26 +434,14 @@ __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v
 // Append one admitted score: reserve a slot, store (kd, idx).  Entries beyond the capacity are
 // counted, not stored.  (The histogram of the refinement digit is built from the compacted
 // on-chip tail right after the pass, see select_adaptive; no second row pass is involved.)
-#if HPCTOPK_EXPERIMENT == 7
-constexpr bool kCount0InScan = true;
-#else
-constexpr bool kCount0InScan = false;   // C(tau_0) is counted from the stored tail after the pass
-#endif
-#ifdef HPCTOPK_WARP_APPEND
-constexpr bool kWarpAppend = true;    // experiment: warp-synchronous slot reservation (measured slower)
-#else
-constexpr bool kWarpAppend = false;
-#endif
-template <bool COUNT0>
+// Measured on this path, and left out because the whole call got slower although fewer
+// instructions ran: storing the raw bits and forming the key when an entry is read; loops
+// specialised on the sign of the cutoff (one compare instead of xor + compare); one atomic per
+// lane and register tile; one atomic per warp and tile after a shuffle scan of the lane counts.
 __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const CandCtx& c) {
   Shared& sh = SH();
   const uint32_t kd = kd_of_bits(u);
-  if (COUNT0 && kd <= sh.count0_cut) atomicAdd(&sh.count0, 1u);
-#if HPCTOPK_EXPERIMENT == 2
-  const uint32_t pos = idx & 2047u; sh.cand_count = 3000;
-#else
   const uint32_t pos = atomicAdd(&sh.cand_count, 1u);
-#endif
   if (pos < c.cap_s) CAND()[pos] = make_uint2(kd, idx);
   else if (pos < c.cap) c.spill[pos - c.cap_s] = make_uint2(kd, idx);
 }
@@ -407,9 +452,9 @@ __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const
 //   BAND = true : admit cut_lo < kd <= cut_hi.   (the band of Eq. "rescue-band")
 // Admitted scores are rare (about 1.5 K / L of the row), so the loop spends one compare and one
 // branch per score and leaves everything else to the taken branch.
-template <int THREADS, int U, bool BAND, bool COUNT0 = false>
+template <int THREADS, int U, bool BAND>
 __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
-                                        uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
+                                             uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
   const int tid = threadIdx.x;
   if (e1 <= e0) return;
   const Admit in_hi(cut_hi);
@@ -428,7 +473,7 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
     else if (tid >= 8 && tid - 8 < ntail) e = e1 - ntail + (tid - 8);
     if (e >= 0) {
       const uint32_t u = __float_as_uint(__ldg(scores + e));
-      if (admit(u)) append_candidate<COUNT0>(u, (uint32_t)(e - g0), cc);
+      if (admit(u)) append_candidate(u, (uint32_t)(e - g0), cc);
     }
   }
   const int64_t nvec = (b1 - b0) >> 2;
@@ -441,74 +486,19 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
   auto classify = [&](const float4& f, uint32_t i) {
     const uint32_t u0 = __float_as_uint(f.x), u1 = __float_as_uint(f.y);
     const uint32_t u2 = __float_as_uint(f.z), u3 = __float_as_uint(f.w);
-    if (admit(u0)) append_candidate<COUNT0>(u0, i + 0, cc);
-    if (admit(u1)) append_candidate<COUNT0>(u1, i + 1, cc);
-    if (admit(u2)) append_candidate<COUNT0>(u2, i + 2, cc);
-    if (admit(u3)) append_candidate<COUNT0>(u3, i + 3, cc);
+    if (admit(u0)) append_candidate(u0, i + 0, cc);
+    if (admit(u1)) append_candidate(u1, i + 1, cc);
+    if (admit(u2)) append_candidate(u2, i + 2, cc);
+    if (admit(u3)) append_candidate(u3, i + 3, cc);
   };
-  // The loads are fed from L2: each thread asks for the lines kPrefetchAheadBytes further on,
-  // so DRAM latency is covered by requests that hold no registers.
-  constexpr int PF_VEC = kPrefetchAheadBytes / 16;
-  const float4* const pf_end = vp + nvec;
+  // (Asking the L2 for lines further ahead with prefetch.global.L2 was measured: no gain.)
   auto load_tile = [&](float4 (&buf)[U], const float4* p) {
 #pragma unroll
-    for (int j = 0; j < U; ++j) {
-      buf[j] = __ldcs(p + j * THREADS);
-#if HPCTOPK_EXPERIMENT == 3
-      if (!BAND) {
-        const float4* q = p + j * THREADS + PF_VEC;
-        if (q < pf_end) asm volatile("prefetch.global.L2 [%0];" ::"l"(q));
-      }
-#endif
-    }
+    for (int j = 0; j < U; ++j) buf[j] = __ldcs(p + j * THREADS);
   };
-  // Whole tiles are classified warp-synchronously: every lane counts its admitted scores, one
-  // shuffle scan turns the counts into slot offsets, and one lane reserves the warp's slots with
-  // a single atomic.  (One atomic per admitted score, each waited for by a diverged lane, made
-  // the latency of the taken branch the largest term of the pass.)
-  const int lane = tid & 31;
   auto process_tile = [&](const float4 (&buf)[U], uint32_t ibase) {
-    if (COUNT0 || !kWarpAppend) {
 #pragma unroll
-      for (int j = 0; j < U; ++j) classify(buf[j], ibase + (uint32_t)(j * THREADS * 4));
-      return;
-    }
-    uint32_t n = 0;
-#pragma unroll
-    for (int j = 0; j < U; ++j) {
-      n += admit(__float_as_uint(buf[j].x)) ? 1u : 0u;
-      n += admit(__float_as_uint(buf[j].y)) ? 1u : 0u;
-      n += admit(__float_as_uint(buf[j].z)) ? 1u : 0u;
-      n += admit(__float_as_uint(buf[j].w)) ? 1u : 0u;
-    }
-    if (!__any_sync(0xFFFFFFFFu, n != 0u)) return;
-    uint32_t incl = n;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-      if (lane >= d) incl += up;
-    }
-    uint32_t base = 0;
-    if (lane == 31) base = atomicAdd(&SH().cand_count, incl);
-    base = __shfl_sync(0xFFFFFFFFu, base, 31);
-    if (n == 0u) return;
-    uint32_t pos = base + incl - n;
-    auto put = [&](uint32_t u, uint32_t idx) {
-      if (admit(u)) {
-        const uint2 e = make_uint2(kd_of_bits(u), idx);
-        if (pos < cc.cap_s) CAND()[pos] = e;
-        else if (pos < cc.cap) cc.spill[pos - cc.cap_s] = e;
-        ++pos;
-      }
-    };
-#pragma unroll
-    for (int j = 0; j < U; ++j) {
-      const uint32_t i = ibase + (uint32_t)(j * THREADS * 4);
-      put(__float_as_uint(buf[j].x), i + 0);
-      put(__float_as_uint(buf[j].y), i + 1);
-      put(__float_as_uint(buf[j].z), i + 2);
-      put(__float_as_uint(buf[j].w), i + 3);
-    }
+    for (int j = 0; j < U; ++j) classify(buf[j], ibase + (uint32_t)(j * THREADS * 4));
   };
 
   // Two register tiles: the loads of one are in flight while the other is classified.
@@ -676,14 +666,10 @@ __device__ __forceinline__ void stats_flush(unsigned char* ws) {
   }
 }
 __device__ __forceinline__ void add64(uint64_t* p, uint64_t v) {
-#if HPCTOPK_EXPERIMENT != 4
   atomicAdd(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
-#endif
 }
 __device__ __forceinline__ void max64(uint64_t* p, uint64_t v) {
-#if HPCTOPK_EXPERIMENT != 4
   atomicMax(reinterpret_cast<unsigned long long*>(p), (unsigned long long)v);
-#endif
 }
 __device__ void record_row(const Params& P, int row, int route, int tau, uint32_t c0, uint32_t cfin,
                            uint64_t scanned, uint64_t sampled, uint64_t L) {
@@ -736,20 +722,29 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   }
   __syncthreads();
   DSTAMP(6, ts);
-  if (threadIdx.x < 32) {                       // one warp locates the three bins and looks their cutoffs up
-    const int lane = threadIdx.x;
-    const LaneSums ls = w_lane_sums(sh.hist, lane);
-    uint32_t below, at;
+  {
     int q_hi = (P.K + 2 * s - 1) / (2 * s);
     if (q_hi < 1) q_hi = 1;
     const uint32_t q2 = (uint32_t)((3 * P.K + s - 1) / s);             // second band: sample rank ceil(3K/s)
     const uint32_t quota[4] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi, q2};
-    int tau[4];
-    w_locate_n<4>(sh.hist, ls, quota, lane, tau);
-    (void)below; (void)at;
-    if (tau[3] < 0) tau[3] = tau[1];                                  // view shorter than q2: no second band
-    if (lane < 4) sh.cutd[lane] = g_cut_table[lane == 0 ? tau[0] : (lane == 1 ? tau[1] : (lane == 2 ? tau[2] : tau[3]))];
-    if (lane == 0) { sh.loc_bin[0] = tau[0]; sh.loc_bin[1] = tau[1]; }
+#ifndef HPCTOPK_P1_BLOCK
+    if (threadIdx.x < 32) {
+      const int lane = threadIdx.x;
+      const LaneSums ls = w_lane_sums(sh.hist, lane);
+      int tau[4];
+      w_locate_n<4>(sh.hist, ls, quota, lane, tau);
+      if (lane < 4) sh.loc_bin[lane] = lane == 0 ? tau[0] : (lane == 1 ? tau[1] : (lane == 2 ? tau[2] : tau[3]));
+      __syncwarp();
+    }
+#else
+    locate_n<THREADS, 4>(quota);
+#endif
+    DSTAMP1(0, ts);
+    if (threadIdx.x < 4) {
+      int tau = sh.loc_bin[threadIdx.x];
+      if (tau < 0) tau = sh.loc_bin[1];                                // view shorter than q2: no second band
+      sh.cutd[threadIdx.x] = g_cut_table[tau];
+    }
   }
   __syncthreads();
   DSTAMP(7, ts);
@@ -798,6 +793,7 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
   }
   __syncthreads();
   DSTAMP(1, ts);
+#ifndef HPCTOPK_SA_BLOCK
   if (tid < 32) {
     const LaneSums ls = w_lane_sums(sh.hist, lane);
     uint32_t below0, at0;
@@ -805,6 +801,12 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
     if (lane == 0) { sh.loc_bin[0] = b0; sh.loc_below[0] = below0; sh.loc_at[0] = at0; }
   }
   __syncthreads();
+#else
+  {
+    const uint32_t quota[1] = {K};
+    locate_n<THREADS, 1>(quota);
+  }
+#endif
   const int b = sh.loc_bin[0];
   const uint32_t below = sh.loc_below[0], at = sh.loc_at[0];
   DSTAMP(2, ts);
@@ -971,11 +973,11 @@ __device__ void process_row(const Params& P, int row) {
   }
   const long long t1 = tick();
   const uint64_t sampled = (uint64_t)((L + P.stride - 1) / P.stride);
-  if (threadIdx.x == 0) { sh.cand_count = 0; sh.count0 = 0; sh.count0_cut = sh.cutd[0]; }
+  if (threadIdx.x == 0) { sh.cand_count = 0; sh.count0 = 0; }
   __syncthreads();
-  scan_range<THREADS, U, false, kCount0InScan>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[1], cc);
+  scan_range<THREADS, U, false>(P.scores, g0, g0, g0 + L, 0u, sh.cutd[1], cc);
   __syncthreads();
-  if (!kCount0InScan) count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
+  count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
   const long long t2 = tick();
   finish_sampled_row<THREADS, U>(P, row, g0, L, sh.count0, sh.cand_count, tau_pack, (uint64_t)L, sampled);
   if (threadIdx.x == 0) {
@@ -1017,11 +1019,11 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   // so that an underfilled primary boundary never costs the finisher a second, single-CTA pass.
   uint32_t* rowcnt0 = rowcnt + kSplitRowsMax;
   __syncthreads();
-  if (threadIdx.x == 0) { sh.cand_count = 0; sh.count0 = 0; sh.count0_cut = sh.cutd[0]; }
+  if (threadIdx.x == 0) { sh.cand_count = 0; sh.count0 = 0; }
   __syncthreads();
-  if (usable) scan_range<THREADS, U, false, kCount0InScan>(P.scores, g0, e0, e1, 0u, sh.cutd[1], cc);
+  if (usable) scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, sh.cutd[1], cc);
   __syncthreads();
-  if (usable && !kCount0InScan) count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
+  if (usable) count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
   const uint32_t Cp = sh.cand_count;
   const long long t2 = tick();
   if (threadIdx.x == 0) {
@@ -1095,11 +1097,7 @@ __device__ __forceinline__ void prefetch_head(const Params& P, int64_t e0, int64
 // Unsplit calls hand rows out from the end of the batch: causal prefill lists rows by growing
 // length, so this runs the longest rows first and leaves short ones to fill the tail of the grid.
 __device__ __forceinline__ int row_of_task(const Params& P, uint32_t task) {
-#if HPCTOPK_EXPERIMENT == 6
-  return (int)task;
-#else
   return P.num_rows - 1 - (int)task;
-#endif
 }
 
 template <int THREADS, int U, int MINB>
@@ -1230,6 +1228,8 @@ const Variant kVariants[] = {
     {hpctopk_kernel<512, 1, 3>, 512},
     {hpctopk_kernel<1024, 1, 1>, 1024},
     {hpctopk_kernel<1024, 2, 1>, 1024},
+    {hpctopk_kernel<448, 2, 3>, 448},
+    {hpctopk_kernel<384, 2, 3>, 384},
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 // 0 selects the warp-specialised kernel, v >= 1 the single-role kernel kVariants[v - 1].
