@@ -30,7 +30,7 @@ K = 2048
 # DRAM bytes per score element of the dominant kernel, from the ncu capture summarised in
 # profiles/hpctopk_kernel_config3_small.md (dram__bytes_read.sum + dram__bytes_write.sum over
 # the valid elements of the captured launch; traffic grows in proportion to the elements).
-NCU_DRAM_BYTES_PER_ELEMENT = 4.49
+NCU_DRAM_BYTES_PER_ELEMENT = 4.83
 
 
 def load_peaks():
