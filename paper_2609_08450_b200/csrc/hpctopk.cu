@@ -88,7 +88,19 @@ struct Params {
   int32_t stride;
   int32_t q0, q1;
   int32_t split_enabled;
+  // Three-kernel pipeline only (zero otherwise): workspace offsets of the per-row boundary
+  // records, the per-row admitted counts, the per-row candidate ranges and the overflow slices.
+  int64_t pipe_rec_off, pipe_cnt_off, pipe_cand_off, pipe_spill_off;
 };
+
+// What the boundary kernel leaves for a row and the other two kernels read.
+struct RowRec {
+  uint32_t cutd[4];          // cutoffs of tau_0, tau_1, tau_hi, tau_2
+  int32_t tau_pack;          // tau_0 | tau_1 << 16, or -1
+  uint32_t usable;           // 1: sampled row with a usable view
+  uint32_t pad[2];
+};
+static_assert(sizeof(RowRec) == 32, "RowRec is read as two 16-byte vectors");
 
 struct Shared {
   hpctopk_stats acc;         // this CTA's counters (first member of every kernel's shared state)
@@ -98,6 +110,7 @@ struct Shared {
   uint32_t out_count;
   uint32_t small_count;
   uint32_t count0;           // C(tau_0) within the stored nested tail
+  uint32_t min_bin;          // Phase 1: smallest occupied coarse bin of the view
   int32_t loc_bin[4];
   uint32_t loc_below[4];
   uint32_t loc_at[4];
@@ -338,12 +351,14 @@ __device__ void locate(Shared& sh, uint32_t quota0, uint32_t quota1, int nq) {
 // (A single warp walking the histogram takes 13 K to 18 K cycles per row next to streaming CTAs,
 // against about 6 K here, yet the whole call ran 3 % slower with this form: the idle warps of the
 // single-warp search cost nothing, the fifteen extra warps here take issue slots from the CTAs
-// that are streaming.  Kept for tuning runs: -DHPCTOPK_P1_BLOCK, -DHPCTOPK_SA_BLOCK.)
+// that are streaming.  The boundary and refinement kernels of the pipeline, which share the SM
+// with no streaming CTA, use this form: BLOCK_SEARCH = true.)
 template <int THREADS, int N>
 __device__ __forceinline__ void locate_n(const uint32_t (&quota)[N]) {
   Shared& sh = SH();
-  constexpr int BPT = THREADS >= 512 ? 4 : 8;
+  constexpr int BPT = THREADS >= 512 ? 4 : (THREADS >= 256 ? 8 : 16);
   constexpr int NT = kBins / BPT, NW = NT / 32;
+  static_assert(NT <= THREADS, "locate_n needs at least 128 threads");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t h[BPT];
   uint32_t sum = 0;
@@ -407,6 +422,13 @@ struct Admit {
     bound = (int32_t)(cu ^ flip);
   }
   __device__ __forceinline__ bool operator()(uint32_t u) const { return (int32_t)(u ^ flip) >= bound; }
+  __device__ __forceinline__ bool negative() const { return flip != 0u; }
+  template <int MODE>
+  __device__ __forceinline__ bool test(uint32_t u) const {
+    if (MODE == 1) return (int32_t)u >= bound;                       // cutoff positive
+    if (MODE == 2) return u <= ((uint32_t)bound ^ 0x7FFFFFFFu);      // cutoff negative
+    return (*this)(u);
+  }
 };
 
 // Where admitted scores go: shared memory first, then this CTA's global overflow slice.
@@ -417,15 +439,25 @@ struct CandCtx {
 __device__ __forceinline__ CandCtx cand_ctx(const Params& P) {
   const size_t cand_off = align_up(kOffRowInfo + (size_t)P.num_rows * sizeof(hpctopk_row_info), 256);
   const size_t split_rows = P.num_rows < kSplitRowsMax ? P.num_rows : kSplitRowsMax;
-  const size_t spill_off = cand_off + split_rows * (size_t)P.cap * 8;
+  const size_t spill_off = P.pipe_spill_off ? (size_t)P.pipe_spill_off : cand_off + split_rows * (size_t)P.cap * 8;
   CandCtx c;
   c.cap_s = (uint32_t)P.cap_s;
   c.cap = (uint32_t)P.cap;
   c.spill = reinterpret_cast<uint2*>(P.ws + spill_off) + (size_t)blockIdx.x * (size_t)(P.cap - P.cap_s);
   return c;
 }
-__device__ __forceinline__ uint2 cand_load(const CandCtx& c, uint32_t i) {   // (kd, idx)
+#ifdef HPCTOPK_RAW
+constexpr bool kRawEntries = true;     // entries hold the raw bits; the key is formed when an entry is read
+#else
+constexpr bool kRawEntries = false;
+#endif
+__device__ __forceinline__ uint2 cand_raw(const CandCtx& c, uint32_t i) {
   return i < c.cap_s ? CAND()[i] : __ldcg(c.spill + (i - c.cap_s));
+}
+__device__ __forceinline__ uint2 cand_load(const CandCtx& c, uint32_t i) {   // (kd, idx)
+  uint2 e = cand_raw(c, i);
+  if (kRawEntries) e.x = kd_of_bits(e.x);
+  return e;
 }
 __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v) {
   if (i < c.cap_s) CAND()[i] = v; else c.spill[i - c.cap_s] = v;
@@ -437,10 +469,13 @@ __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v
 // Measured on this path, and left out because the whole call got slower although fewer
 // instructions ran: storing the raw bits and forming the key when an entry is read; loops
 // specialised on the sign of the cutoff (one compare instead of xor + compare); one atomic per
-// lane and register tile; one atomic per warp and tile after a shuffle scan of the lane counts.
+// lane and register tile; one atomic per warp and tile after a shuffle scan of the lane counts;
+// one vote per element position with converged stores; one gating branch per vector or tile.
+// (Diverged lanes on this short path run in the shadow of the converged ones; every converged
+// form makes the whole warp wait at its votes and shuffles.)
 __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const CandCtx& c) {
   Shared& sh = SH();
-  const uint32_t kd = kd_of_bits(u);
+  const uint32_t kd = kRawEntries ? u : kd_of_bits(u);
   const uint32_t pos = atomicAdd(&sh.cand_count, 1u);
   if (pos < c.cap_s) CAND()[pos] = make_uint2(kd, idx);
   else if (pos < c.cap) c.spill[pos - c.cap_s] = make_uint2(kd, idx);
@@ -452,14 +487,14 @@ __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const
 //   BAND = true : admit cut_lo < kd <= cut_hi.   (the band of Eq. "rescue-band")
 // Admitted scores are rare (about 1.5 K / L of the row), so the loop spends one compare and one
 // branch per score and leaves everything else to the taken branch.
-template <int THREADS, int U, bool BAND>
-__device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
+template <int THREADS, int U, bool BAND, int MODE>
+__device__ __forceinline__ void scan_body(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
                                              uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
   const int tid = threadIdx.x;
   if (e1 <= e0) return;
   const Admit in_hi(cut_hi);
   const Admit in_lo(cut_lo);                 // BAND: scores admitted by tau_0 are already held
-  auto admit = [&](uint32_t u) -> bool { return BAND ? (in_hi(u) && !in_lo(u)) : in_hi(u); };
+  auto admit = [&](uint32_t u) -> bool { return BAND ? (in_hi(u) && !in_lo(u)) : in_hi.template test<MODE>(u); };
   int64_t b0 = (e0 + 3) & ~(int64_t)3;       // first 16-byte aligned element
   int64_t b1 = e1 & ~(int64_t)3;             // end of the last whole vector
   if (b0 > b1) { b0 = e1; b1 = e1; }         // range holds no whole vector
@@ -521,6 +556,30 @@ __device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_
   for (int64_t v = nfull * TILE + tid; v < nvec; v += THREADS)
     classify(__ldcs(vp + v), idx0 + (uint32_t)(v << 2));
 }
+
+#ifndef HPCTOPK_SIGNSPEC
+template <int THREADS, int U, bool BAND>
+__device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
+                                        uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
+  scan_body<THREADS, U, BAND, 0>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
+}
+#else
+template <int THREADS, int U, bool BAND, int MODE>
+__device__ __noinline__ void scan_range_m(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
+                                          uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
+  scan_body<THREADS, U, BAND, MODE>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
+}
+template <int THREADS, int U, bool BAND>
+__device__ __forceinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
+                                           uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
+  if (!BAND) {                               // one compare per score, by the sign of the cutoff
+    if (Admit(cut_hi).negative()) scan_range_m<THREADS, U, false, 2>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
+    else scan_range_m<THREADS, U, false, 1>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
+    return;
+  }
+  scan_range_m<THREADS, U, BAND, 0>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
+}
+#endif
 
 // ---------------------------------------------------------------- element sources for selection
 // A source visits every element once per pass, calling f(valid, kd, idx) with a block-uniform
@@ -692,7 +751,7 @@ __device__ void record_row(const Params& P, int row, int route, int tau, uint32_
 // A third, tighter bin tau_hi at half the rank K (sample rank ceil(K / 2s)) brackets the K-th
 // score from above; its cutoff sizes the refinement digit of select_adaptive.
 // Returns false when the view cannot support the requested sample ranks.
-template <int THREADS>
+template <int THREADS, bool BLOCK_SEARCH = false>
 __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_t L, int& tau_pack) {
   Shared& sh = SH();
   const int s = P.stride;
@@ -704,8 +763,10 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   long long ts = tick();
   __syncthreads();
   clear_hist<THREADS>(sh);
+  if (threadIdx.x == 0) sh.min_bin = kBins - 1;
   __syncthreads();
   DSTAMP(5, ts);
+  uint32_t my_min = kBins - 1;
   const float* __restrict__ rowp = P.scores + g0 + a;
   for (int64_t t0 = 0; t0 < n_view; t0 += 4 * THREADS) {
     uint32_t u[4];
@@ -714,12 +775,20 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
     for (int k = 0; k < 4; ++k) {
       const int64_t t = t0 + k * THREADS + threadIdx.x;
       v[k] = t < n_view;
-      u[k] = v[k] ? __float_as_uint(__ldg(rowp + t * s)) : 0u;
+      // no L1 line, 64-byte L2 fetch: the default 128-byte fetch doubles the DRAM traffic of the view
+      u[k] = 0u;
+      if (v[k]) asm volatile("ld.global.nc.L1::no_allocate.L2::64B.b32 %0, [%1];" : "=r"(u[k]) : "l"(rowp + t * s));
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k)
-      if (v[k]) atomicAdd(&sh.hist[coarse_bin_of_kd(kd_of_bits(u[k]))], 1u);
+      if (v[k]) {
+        const uint32_t bin = (uint32_t)coarse_bin_of_kd(kd_of_bits(u[k]));
+        atomicAdd(&sh.hist[bin], 1u);
+        my_min = bin < my_min ? bin : my_min;
+      }
   }
+  my_min = __reduce_min_sync(0xFFFFFFFFu, my_min);
+  if ((threadIdx.x & 31) == 0 && my_min < kBins - 1) atomicMin(&sh.min_bin, my_min);
   __syncthreads();
   DSTAMP(6, ts);
   {
@@ -727,18 +796,37 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
     if (q_hi < 1) q_hi = 1;
     const uint32_t q2 = (uint32_t)((3 * P.K + s - 1) / s);             // second band: sample rank ceil(3K/s)
     const uint32_t quota[4] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi, q2};
-#ifndef HPCTOPK_P1_BLOCK
+    // The four sample ranks are all small (at most 3K/s of the n_view samples), so their bins lie
+    // within a few dozen bins of the best occupied one: one warp walks the histogram upwards from
+    // there, 32 bins per step, instead of forming the prefix of all 2048 bins.
     if (threadIdx.x < 32) {
       const int lane = threadIdx.x;
-      const LaneSums ls = w_lane_sums(sh.hist, lane);
-      int tau[4];
-      w_locate_n<4>(sh.hist, ls, quota, lane, tau);
+      int tau[4] = {-1, -1, -1, -1};
+      uint32_t carry = 0;
+      for (int base = (int)(sh.min_bin & ~31u); base < kBins; base += 32) {
+        const uint32_t h = sh.hist[base + lane];
+        uint32_t incl = h;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+          if (lane >= d) incl += up;
+        }
+        const uint32_t cum = carry + incl;
+        bool all = true;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (tau[k] < 0) {
+            const uint32_t m = __ballot_sync(0xFFFFFFFFu, cum >= quota[k]);
+            if (m) tau[k] = base + __ffs(m) - 1;
+          }
+          all = all && tau[k] >= 0;
+        }
+        if (all) break;
+        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      }
       if (lane < 4) sh.loc_bin[lane] = lane == 0 ? tau[0] : (lane == 1 ? tau[1] : (lane == 2 ? tau[2] : tau[3]));
       __syncwarp();
     }
-#else
-    locate_n<THREADS, 4>(quota);
-#endif
     DSTAMP1(0, ts);
     if (threadIdx.x < 4) {
       int tau = sh.loc_bin[threadIdx.x];
@@ -760,9 +848,9 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
 // ranking its members against each other under (kd, idx).  Returns false, with nothing written,
 // when the K-th score falls outside the bracket or the boundary bin is too large: the caller
 // then runs the general 11+11+10 refinement.
-template <int THREADS>
+template <int THREADS, bool BLOCK_SEARCH = false, bool COUNT0 = false>
 __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint32_t K, uint32_t cut_base, uint32_t cut_hi,
-                                             int32_t* out_idx, float* out_val) {
+                                             int32_t* out_idx, float* out_val, uint32_t cut_count = 0u) {
   Shared& sh = SH();
   const int tid = threadIdx.x, lane = tid & 31;
   const uint32_t span = cut_base > cut_hi ? cut_base - cut_hi : 0u;
@@ -779,6 +867,7 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
   if (tid == 0) { sh.out_count = 0; sh.small_count = 0; }
   __syncthreads();
   DSTAMP(0, ts);
+  uint32_t n0 = 0;                               // COUNT0: entries with kd <= cut_count, added to sh.count0
   for (uint32_t i0 = 0; i0 < C; i0 += 4 * THREADS) {
     uint2 c[4];
     bool v[4];
@@ -787,13 +876,18 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
       const uint32_t i = i0 + k * THREADS + tid;
       c[k] = i < C ? cand_load(cc, i) : make_uint2(0xFFFFFFFFu, 0u);
       v[k] = i < C && c[k].x <= cut_base;       // a split row's buffer also holds the band beyond tau_0
+      if (COUNT0) n0 += (i < C && c[k].x <= cut_count) ? 1u : 0u;
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k) if (v[k]) atomicAdd(&sh.hist[digit(c[k].x)], 1u);
   }
+  if (COUNT0) {
+    n0 = __reduce_add_sync(0xFFFFFFFFu, n0);
+    if (lane == 0 && n0) atomicAdd(&sh.count0, n0);
+  }
   __syncthreads();
   DSTAMP(1, ts);
-#ifndef HPCTOPK_SA_BLOCK
+  if (!BLOCK_SEARCH) {
   if (tid < 32) {
     const LaneSums ls = w_lane_sums(sh.hist, lane);
     uint32_t below0, at0;
@@ -801,12 +895,10 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
     if (lane == 0) { sh.loc_bin[0] = b0; sh.loc_below[0] = below0; sh.loc_at[0] = at0; }
   }
   __syncthreads();
-#else
-  {
+  } else {
     const uint32_t quota[1] = {K};
     locate_n<THREADS, 1>(quota);
   }
-#endif
   const int b = sh.loc_bin[0];
   const uint32_t below = sh.loc_below[0], at = sh.loc_at[0];
   DSTAMP(2, ts);
@@ -892,11 +984,10 @@ __device__ __forceinline__ void count_primary(const CandCtx& cc, uint32_t n, uin
 // all of them.  A row that is still underfilled appends one wider band (tau_1, tau_2] in a
 // second pass before it falls back to the storage-free recovery.  On entry the candidate arrays
 // hold min(C1, cap) entries and sh.cand_count == C1.
-template <int THREADS, int U>
-__device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t L, uint32_t C0, uint32_t C1,
-                                   int tau_pack, uint64_t scanned, uint64_t sampled) {
+template <int THREADS, int U, bool BLOCK_SEARCH = false>
+__device__ void finish_sampled_row(const Params& P, const CandCtx cc, int row, int64_t g0, int64_t L, uint32_t C0,
+                                   uint32_t C1, int tau_pack, uint64_t scanned, uint64_t sampled) {
   Shared& sh = SH();
-  const CandCtx cc = cand_ctx(P);
   int32_t* oi = P.out_idx + (int64_t)row * P.K;
   float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
   const uint32_t K = (uint32_t)P.K, cap = (uint32_t)P.cap;
@@ -920,7 +1011,7 @@ __device__ void finish_sampled_row(const Params& P, int row, int64_t g0, int64_t
     }
   }
   if (cfin) {
-    if (!select_adaptive<THREADS>(cc, C, K, cut_base, sh.cutd[2], oi, ov)) {
+    if (!select_adaptive<THREADS, BLOCK_SEARCH>(cc, C, K, cut_base, sh.cutd[2], oi, ov)) {
       if (threadIdx.x == 0) add64(&stats_of(P.ws)->general_refinements, 1);
       __syncthreads();
       CandidateSource cs{cc, C, cut_base};
@@ -979,7 +1070,7 @@ __device__ void process_row(const Params& P, int row) {
   __syncthreads();
   count_primary<THREADS>(cc, sh.cand_count < cap ? sh.cand_count : cap, sh.cutd[0]);
   const long long t2 = tick();
-  finish_sampled_row<THREADS, U>(P, row, g0, L, sh.count0, sh.cand_count, tau_pack, (uint64_t)L, sampled);
+  finish_sampled_row<THREADS, U>(P, cc, row, g0, L, sh.count0, sh.cand_count, tau_pack, (uint64_t)L, sampled);
   if (threadIdx.x == 0) {
     hpctopk_stats* st = stats_of(P.ws);
     add64(&st->cycles_phase1, (uint64_t)(t1 - t0));
@@ -1038,7 +1129,7 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   __syncthreads();
   const uint32_t base = sh.bcast0;
   if (base + Cp <= cap) {
-    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gcand[base + i] = cand_load(cc, i);
+    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gcand[base + i] = cand_raw(cc, i);
   }
   __threadfence();
   __syncthreads();
@@ -1063,7 +1154,7 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   }
   if (threadIdx.x == 0) sh.cand_count = C1;
   __syncthreads();
-  finish_sampled_row<THREADS, U>(P, row, g0, L, C0, C1, tau_pack, 0, 0);
+  finish_sampled_row<THREADS, U>(P, cc, row, g0, L, C0, C1, tau_pack, 0, 0);
   if (threadIdx.x == 0) add64(&stats_of(P.ws)->cycles_finish, (uint64_t)(tick() - t2));
 }
 
@@ -1100,6 +1191,57 @@ __device__ __forceinline__ int row_of_task(const Params& P, uint32_t task) {
   return P.num_rows - 1 - (int)task;
 }
 
+// Device-side ragged dispatch (Section 4.5): every CTA derives the same task table from
+// row_lengths.  seg_base[r] is the first task of row r, seg_base[num_rows] the task count; a long
+// row gets ceil(L / S) segment tasks with S = max(16384, total / (grid * kTasksPerCta)) rounded
+// up to 4096 elements, every other row one task.  Contains block barriers.
+template <int THREADS>
+__device__ uint32_t build_task_table(const Params& P, uint32_t* seg_base) {
+  Shared& sh = SH();
+  const int tid = threadIdx.x;
+  constexpr int RPT = (kSplitRowsMax + THREADS - 1) / THREADS;
+  unsigned long long mine = 0;
+  for (int j = 0; j < RPT; ++j) {
+    const int r = tid * RPT + j;
+    if (r < P.num_rows) { const int64_t L = P.row_lengths[r]; if (L > P.cap) mine += (unsigned long long)L; }
+  }
+  for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
+  if ((tid & 31) == 0) { sh.hist[2 * (tid >> 5)] = (uint32_t)mine; sh.hist[2 * (tid >> 5) + 1] = (uint32_t)(mine >> 32); }
+  __syncthreads();
+  unsigned long long total = 0;
+  for (int w = 0; w < THREADS / 32; ++w) total += (unsigned long long)sh.hist[2 * w] | ((unsigned long long)sh.hist[2 * w + 1] << 32);
+  const unsigned long long target = (unsigned long long)gridDim.x * kTasksPerCta;
+  unsigned long long S = (total + target - 1) / target;
+  if (S < (unsigned long long)kSegMinElems) S = kSegMinElems;
+  S = (S + 4095ull) / 4096ull * 4096ull;
+  __syncthreads();
+  uint32_t cnt[RPT];
+  uint32_t sum = 0;
+  for (int j = 0; j < RPT; ++j) {
+    const int r = tid * RPT + j;
+    cnt[j] = 0;
+    if (r < P.num_rows) {
+      const int64_t L = P.row_lengths[r];
+      cnt[j] = (L > P.cap) ? (uint32_t)((L + (int64_t)S - 1) / (int64_t)S) : 1u;
+    }
+    sum += cnt[j];
+  }
+  const uint32_t incl = warp_inclusive_scan<THREADS>(sum);
+  if ((tid & 31) == 31) sh.warp_sums[tid >> 5] = incl;
+  __syncthreads();
+  uint32_t woff = 0;
+  for (int w = 0; w < (tid >> 5); ++w) woff += sh.warp_sums[w];
+  uint32_t run = woff + incl - sum;
+  for (int j = 0; j < RPT; ++j) {
+    const int r = tid * RPT + j;
+    if (r < P.num_rows) seg_base[r] = run;
+    run += cnt[j];
+    if (r == P.num_rows - 1) { seg_base[P.num_rows] = run; sh.total_tasks = run; }
+  }
+  __syncthreads();
+  return sh.total_tasks;
+}
+
 template <int THREADS, int U, int MINB>
 __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) {
   Shared& sh = SH();
@@ -1110,50 +1252,7 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
   stats_clear();
   __syncthreads();
   uint32_t total_tasks = (uint32_t)P.num_rows;
-  if (P.split_enabled) {
-    // Device-side ragged dispatch: every CTA derives the same task table from row_lengths.
-    constexpr int RPT = (kSplitRowsMax + THREADS - 1) / THREADS;
-    unsigned long long mine = 0;
-    for (int j = 0; j < RPT; ++j) {
-      const int r = tid * RPT + j;
-      if (r < P.num_rows) { const int64_t L = P.row_lengths[r]; if (L > P.cap) mine += (unsigned long long)L; }
-    }
-    for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
-    if ((tid & 31) == 0) { sh.hist[2 * (tid >> 5)] = (uint32_t)mine; sh.hist[2 * (tid >> 5) + 1] = (uint32_t)(mine >> 32); }
-    __syncthreads();
-    unsigned long long total = 0;
-    for (int w = 0; w < THREADS / 32; ++w) total += (unsigned long long)sh.hist[2 * w] | ((unsigned long long)sh.hist[2 * w + 1] << 32);
-    const unsigned long long target = (unsigned long long)gridDim.x * kTasksPerCta;
-    unsigned long long S = (total + target - 1) / target;
-    if (S < (unsigned long long)kSegMinElems) S = kSegMinElems;
-    S = (S + 4095ull) / 4096ull * 4096ull;
-    __syncthreads();
-    uint32_t cnt[RPT];
-    uint32_t sum = 0;
-    for (int j = 0; j < RPT; ++j) {
-      const int r = tid * RPT + j;
-      cnt[j] = 0;
-      if (r < P.num_rows) {
-        const int64_t L = P.row_lengths[r];
-        cnt[j] = (L > P.cap) ? (uint32_t)((L + (int64_t)S - 1) / (int64_t)S) : 1u;
-      }
-      sum += cnt[j];
-    }
-    const uint32_t incl = warp_inclusive_scan<THREADS>(sum);
-    if ((tid & 31) == 31) sh.warp_sums[tid >> 5] = incl;
-    __syncthreads();
-    uint32_t woff = 0;
-    for (int w = 0; w < (tid >> 5); ++w) woff += sh.warp_sums[w];
-    uint32_t run = woff + incl - sum;
-    for (int j = 0; j < RPT; ++j) {
-      const int r = tid * RPT + j;
-      if (r < P.num_rows) seg_base[r] = run;
-      run += cnt[j];
-      if (r == P.num_rows - 1) { seg_base[P.num_rows] = run; sh.total_tasks = run; }
-    }
-    __syncthreads();
-    total_tasks = sh.total_tasks;
-  }
+  if (P.split_enabled) total_tasks = build_task_table<THREADS>(P, seg_base);
 
   // Two statically assigned waves, then completion-order claiming from the device counter.
   // The claim for the task after next is issued at the top of each task, so its latency and the
@@ -1191,6 +1290,229 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
     next = claimed;
   }
   __syncthreads();
+  if (tid == 0) stats_flush(P.ws);
+}
+
+
+// ---------------------------------------------------------------- the three-kernel pipeline
+// The same steps as hpctopk_kernel, cut at the two points where a row's CTA would otherwise stop
+// streaming: (1) boundary kernel, Phase 1 of every sampled row; (2) pass kernel, nothing but
+// complete-row passes, each leaving its admitted tail in the row's global candidate range;
+// (3) refinement kernel, certification branch, Phase 3 and the output commit of every row.
+// In the single kernel a CTA streams for about half of its time (Phase 1 and Phase 3 hold its
+// registers and shared memory while its loads are stopped); here the pass kernel streams all the
+// time and the short phases run at their own, higher occupancy.  Cost: the admitted tails cross
+// HBM once each way (about 57 KB per row at K = 2048, 11 % of a 129 K-score row).
+constexpr uint32_t kBand2Flag = 0x80000000u;    // in a row's admitted count: the tail includes the second band
+__device__ __forceinline__ RowRec* pipe_rec(const Params& P) { return reinterpret_cast<RowRec*>(P.ws + P.pipe_rec_off); }
+__device__ __forceinline__ uint32_t* pipe_cnt(const Params& P) { return reinterpret_cast<uint32_t*>(P.ws + P.pipe_cnt_off); }
+__device__ __forceinline__ uint2* pipe_cand(const Params& P, int row) {
+  return reinterpret_cast<uint2*>(P.ws + P.pipe_cand_off) + (size_t)row * (size_t)P.cap;
+}
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) pipe_boundary_kernel(const Params P) {
+  Shared& sh = SH();
+  stats_clear();
+  __syncthreads();
+  for (int row = blockIdx.x; row < P.num_rows; row += gridDim.x) {
+    const int64_t g0 = P.row_starts[row];
+    const int64_t L = P.row_lengths[row];
+    int tau_pack = -1;
+    bool usable = false;
+    if (L > (int64_t)P.cap) usable = phase1<THREADS, true>(P, row, g0, L, tau_pack);
+    __syncthreads();
+    RowRec* rec = pipe_rec(P) + row;
+    if (threadIdx.x < 4) rec->cutd[threadIdx.x] = usable ? sh.cutd[threadIdx.x] : 0u;
+    if (threadIdx.x == 0) {
+      rec->tau_pack = tau_pack;
+      rec->usable = usable ? 1u : 0u;
+      pipe_cnt(P)[row] = 0u;
+    }
+    __syncthreads();
+  }
+}
+
+// One task of the pass kernel: elements [e0, e1) of a sampled row.
+template <int THREADS, int U>
+__device__ void pipe_pass_task(const Params& P, int row, int seg, int nseg) {
+  Shared& sh = SH();
+  const CandCtx cc = cand_ctx(P);
+  const int64_t g0 = P.row_starts[row];
+  const int64_t L = P.row_lengths[row];
+  if (L <= (int64_t)P.cap) return;                       // short and direct rows: refinement kernel
+  const RowRec* rec = pipe_rec(P) + row;
+  const uint4 r0 = __ldg(reinterpret_cast<const uint4*>(rec));
+  const uint4 r1 = __ldg(reinterpret_cast<const uint4*>(rec) + 1);
+  if (r1.y == 0u) return;                                // unusable view: refinement kernel recovers
+  const uint32_t cut1 = r0.y, cap = (uint32_t)P.cap;
+  const int64_t g1 = g0 + L;
+  int64_t e0 = g0, e1 = g1;
+  if (nseg > 1) {                                        // contiguous, 16-byte aligned partition
+    const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
+    const int64_t per = (vb - va + nseg - 1) / nseg;
+    e0 = (va + (int64_t)seg * per) << 2;
+    e1 = (va + (int64_t)(seg + 1) * per) << 2;
+    if (e0 < g0) e0 = g0;
+    if (e1 > g1) e1 = g1;
+    if (e1 < e0) e1 = e0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) sh.cand_count = 0;
+  __syncthreads();
+  scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, cut1, cc);
+  __syncthreads();
+  uint32_t Cp = sh.cand_count;
+  uint32_t flag = 0u;
+  uint64_t scanned = (uint64_t)(e1 - e0);
+  if (nseg == 1 && Cp < (uint32_t)P.K && r0.w > cut1) {
+    // Underfilled row owned by this CTA: append the second band (tau_1, tau_2] here, where the
+    // row has just passed through the L2 and 16 warps stream it, and tell the refinement kernel.
+    __syncthreads();
+    scan_range<THREADS, U, true>(P.scores, g0, g0, g1, cut1, r0.w, cc);
+    __syncthreads();
+    Cp = sh.cand_count;
+    flag = kBand2Flag;
+    scanned += (uint64_t)L;
+  }
+  if (threadIdx.x == 0) {
+    sh.bcast0 = atomicAdd(&pipe_cnt(P)[row], Cp | flag) & ~kBand2Flag;
+    hpctopk_stats* st = stats_of(P.ws);
+    add64(&st->elements_scanned, scanned);
+    if (nseg > 1 && seg == 0) add64(&st->rows_split, 1);
+  }
+  __syncthreads();
+  const uint32_t base = sh.bcast0;
+  if (Cp <= cap && base + Cp <= cap) {                   // otherwise the row total exceeds the capacity anyway
+    uint2* gc = pipe_cand(P, row) + base;
+    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gc[i] = cand_raw(cc, i);
+  }
+}
+
+template <int THREADS, int U, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB) pipe_pass_kernel(const Params P) {
+  Shared& sh = SH();
+  uint32_t* const seg_base = reinterpret_cast<uint32_t*>(CAND() + P.cap_s);   // [kSplitRowsMax + 1], only when splitting
+  uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl);
+  const int tid = threadIdx.x;
+  stats_clear();
+  __syncthreads();
+  uint32_t total_tasks = (uint32_t)P.num_rows;
+  if (P.split_enabled) total_tasks = build_task_table<THREADS>(P, seg_base);
+  uint32_t task = blockIdx.x;
+  uint32_t next = blockIdx.x + gridDim.x;
+  while (task < total_tasks) {
+    if (tid == 0) sh.claim = (int32_t)(2u * gridDim.x + atomicAdd(task_counter, 1u));
+#ifdef HPCTOPK_PASS_PREFETCH
+    if (!P.split_enabled && next < total_tasks) {
+      const int nrow = row_of_task(P, next);
+      const int64_t ng0 = P.row_starts[nrow], nL = P.row_lengths[nrow];
+      if (nL > P.cap) prefetch_head<THREADS>(P, ng0, ng0 + nL);
+    }
+#endif
+    if (P.split_enabled) {
+      int lo = 0, hi = P.num_rows - 1;
+      while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (seg_base[mid] <= task) lo = mid; else hi = mid - 1; }
+      pipe_pass_task<THREADS, U>(P, lo, (int)(task - seg_base[lo]), (int)(seg_base[lo + 1] - seg_base[lo]));
+    } else {
+      pipe_pass_task<THREADS, U>(P, row_of_task(P, task), 0, 1);
+    }
+    __syncthreads();
+    const uint32_t claimed = (uint32_t)sh.claim;
+    if (tid == 0) add64(&stats_of(P.ws)->tasks, 1);
+    __syncthreads();
+    task = next;
+    next = claimed;
+  }
+  __syncthreads();
+  if (tid == 0) stats_flush(P.ws);
+}
+
+// The refinement kernel keeps no candidates on chip: it reads a row's admitted tail from its
+// global range (L2 for the most part, the pass kernel has just written it), so a CTA needs only
+// the 8 KB histogram and many rows are in flight per SM; the refinement is a chain of short
+// dependent steps and is bound by latency, not by bandwidth.  P.cap_s is 0 in this launch: the
+// rare rows that need a staging area (direct rows, second band) use the CTA's global slice.
+template <int THREADS, int U, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params P) {
+  Shared& sh = SH();
+  uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl) + 1;
+  const int tid = threadIdx.x;
+  const uint32_t cap = (uint32_t)P.cap, K = (uint32_t)P.K;
+  stats_clear();
+  __syncthreads();
+  long long t_life = tick();
+#if HPCTOPK_TIMERS
+  unsigned long long gt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0));
+#endif
+  // Every row is claimed from the device counter, the first one too: a CTA that becomes resident
+  // late (the grid may exceed what the SMs hold at once) then finds the rows already taken
+  // instead of sitting on a statically assigned one.
+  if (tid == 0) sh.claim = (int32_t)atomicAdd(task_counter, 1u);
+  __syncthreads();
+  uint32_t task = (uint32_t)sh.claim;
+  __syncthreads();
+  while (task < (uint32_t)P.num_rows) {
+    long long ts = tick();
+    if (tid == 0) sh.claim = (int32_t)atomicAdd(task_counter, 1u);
+    const int row = row_of_task(P, task);
+    const int64_t g0 = P.row_starts[row];
+    const int64_t L = P.row_lengths[row];
+    const RowRec* rec = pipe_rec(P) + row;
+    const bool sampled = L > (int64_t)cap && __ldg(&rec->usable) != 0u;
+    if (!sampled) {
+      process_row<THREADS, U>(P, row);                   // short, direct, or recovery of an unusable view
+    } else {
+      __syncthreads();
+      if (tid < 4) sh.cutd[tid] = __ldg(&rec->cutd[tid]);
+      const int tau_pack = __ldg(&rec->tau_pack);
+      const uint32_t cnt = __ldcg(&pipe_cnt(P)[row]);
+      const bool band2 = (cnt & kBand2Flag) != 0u;
+      const uint32_t C1 = cnt & ~kBand2Flag;             // entries of A(tau_1), or of A(tau_2) with the flag
+      if (tid == 0) { sh.cand_count = C1; sh.count0 = 0; }
+      __syncthreads();
+      CandCtx rc;                                        // the row's global candidate range
+      rc.cap_s = 0u; rc.cap = cap; rc.spill = pipe_cand(P, row);
+      const uint64_t sampled_n = (uint64_t)((L + P.stride - 1) / P.stride);
+      int32_t* oi = P.out_idx + (int64_t)row * P.K;
+      float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
+      if (C1 >= K && C1 <= cap) {
+        // The K best of a larger nested tail are the K best of every smaller one that holds K
+        // entries, so the whole stored tail is refined against its own cutoff and C(tau_0) is
+        // only counted (for the route the row reports).
+        const uint32_t cut_base = band2 ? sh.cutd[3] : sh.cutd[1];
+        if (!select_adaptive<THREADS, true, true>(rc, C1, K, cut_base, sh.cutd[2], oi, ov, sh.cutd[0])) {
+          if (tid == 0) add64(&stats_of(P.ws)->general_refinements, 1);
+          __syncthreads();
+          CandidateSource cs{rc, C1, cut_base};
+          select_and_emit<THREADS>(cs, K, false, oi, ov);
+        }
+        const uint32_t C0 = sh.count0;
+        const int route = band2 ? HPCTOPK_ROUTE_BAND2 : (C0 >= K ? HPCTOPK_ROUTE_PRIMARY : HPCTOPK_ROUTE_BAND);
+        record_row(P, row, route, tau_pack, C0, route == HPCTOPK_ROUTE_PRIMARY ? C0 : C1, 0, sampled_n, (uint64_t)L);
+      } else if (!band2) {
+        // a split row that is still short, or a tail beyond the capacity: the general branch
+        count_primary<THREADS>(rc, C1 <= cap ? C1 : 0u, sh.cutd[0]);
+        finish_sampled_row<THREADS, U, true>(P, rc, row, g0, L, sh.count0, C1, tau_pack, 0, sampled_n);
+      } else {
+        // the second band was tried by the pass kernel and did not certify the row
+        count_primary<THREADS>(rc, C1 <= cap ? C1 : 0u, sh.cutd[0]);
+        RowSource rs{P.scores, g0, g0 + L};
+        select_and_emit<THREADS>(rs, K, false, oi, ov);
+        record_row(P, row, C1 > cap ? HPCTOPK_ROUTE_OVERFLOW : HPCTOPK_ROUTE_RECOVERY, tau_pack, sh.count0, 0,
+                   4ull * (uint64_t)L, sampled_n, (uint64_t)L);
+      }
+    }
+    __syncthreads();
+    const uint32_t claimed = (uint32_t)sh.claim;
+    __syncthreads();
+    task = claimed;
+  }
+  __syncthreads();
+  DSTAMP(5, t_life);
+#if HPCTOPK_TIMERS
+  if (tid == 0) { unsigned long long gt1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1)); atomicAdd(reinterpret_cast<unsigned long long*>(&stats_of(nullptr)->cycles_detail[7]), gt1 - gt0); atomicMax(reinterpret_cast<unsigned long long*>(&stats_of(nullptr)->candidates_max), gt1 - gt0); }
+#endif
   if (tid == 0) stats_flush(P.ws);
 }
 
@@ -1233,8 +1555,19 @@ const Variant kVariants[] = {
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 // 0 selects the warp-specialised kernel, v >= 1 the single-role kernel kVariants[v - 1].
-constexpr int kDefaultVariant = 4;
+// kPipeVariant selects the three-kernel pipeline (calls of at most kPipeRowsMax rows; larger calls
+// use the single kernel, whose workspace does not grow with the row count).
+constexpr int kPipeVariant = 200;
+constexpr int kDefaultVariant = kPipeVariant;
+constexpr int kMonoVariant = 4;
 constexpr int kSplitVariant = 1;
+constexpr int kPipeRowsMax = 8192;
+constexpr int kBoundaryThreads = 128;
+#ifndef HPCTOPK_REFINE_T
+#define HPCTOPK_REFINE_T 128
+#define HPCTOPK_REFINE_MINB 8
+#endif
+constexpr int kRefineThreads = HPCTOPK_REFINE_T;
 constexpr int kFusedVariant = 100;     // single-role kernel with warp-synchronous compaction (namespace wsf)
 
 struct DeviceInfo {
@@ -1242,6 +1575,9 @@ struct DeviceInfo {
   int sm_count = 0;
   int variant = 0;      // 0: warp-specialised kernel; v >= 1: single-role kernel kVariants[v - 1]
   int ctas_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // [split][capacity class]
+  int pass_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // pipeline: pass kernel
+  int refine_per_sm[3] = {0, 0, 0};                 // pipeline: refinement kernel
+  int boundary_per_sm = 0;                          // pipeline: boundary kernel
 };
 DeviceInfo g_dev[64];
 
@@ -1254,13 +1590,36 @@ size_t smem_bytes_for(int cap_s, bool split) {
 // Index into kVariants for a call: calls with few rows (split mode) are latency-bound and
 // prefer fewer, fatter CTAs per SM than the streaming default.
 int variant_index(int variant, bool split) {
-  const int v = (variant == kDefaultVariant && split) ? kSplitVariant : variant;
+  if (variant == kPipeVariant) variant = kMonoVariant;
+  const int v = (variant == kMonoVariant && split) ? kSplitVariant : variant;
   return (v > 0 && v <= kNumVariants) ? v - 1 : 0;
 }
 
 // Shared memory is sized by capacity class so that occupancy (and the grid) depends on K only.
 int cap_class(int K) { return K <= 1024 ? 0 : (K <= 2048 ? 1 : 2); }
 int class_cap_s(int cls) { return smem_capacity_for(cls == 0 ? 1024 : (cls == 1 ? 2048 : HPCTOPK_MAX_K)); }
+
+// Workspace layout of the pipeline: the common head (control block, counters, row records of
+// hpctopk_read_row_info), then boundary records, admitted counts, one candidate range of
+// `capacity` entries per row, and the overflow slices.
+struct PipeLayout { size_t rec, cnt, cand, spill, total; };
+PipeLayout pipe_layout(int rows, int K) {
+  const size_t cap = (size_t)capacity_for(K);
+  const int cap_s_cls = class_cap_s(cap_class(K));
+  const size_t cap_s = (size_t)cap_s_cls < cap ? (size_t)cap_s_cls : cap;
+  PipeLayout l;
+  l.rec = align_up(kOffRowInfo + (size_t)rows * sizeof(hpctopk_row_info), 256);
+  l.cnt = align_up(l.rec + (size_t)rows * sizeof(RowRec), 256);
+  l.cand = align_up(l.cnt + (size_t)rows * sizeof(uint32_t), 256);
+  l.spill = l.cand + (size_t)rows * cap * 8;
+  l.total = align_up(l.spill + (size_t)kMaxGrid * cap * 8, 256);   // the refinement kernel stages nothing on chip
+  return l;
+}
+
+const auto kPassKernel = pipe_pass_kernel<512, 2, 3>;
+constexpr int kPassThreads = 512;
+const auto kRefineKernel = pipe_refine_kernel<kRefineThreads, 2, HPCTOPK_REFINE_MINB>;
+const auto kBoundaryKernel = pipe_boundary_kernel<kBoundaryThreads>;
 
 }  // namespace
 
@@ -1295,7 +1654,12 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
   const size_t spill_wf = wsf::ws_spill_bytes(K, kMaxGrid);
   if (spill_wf > spill) spill = spill_wf;
   b += spill;
-  return align_up(b, 256);
+  b = align_up(b, 256);
+  if (max_num_rows <= kPipeRowsMax) {
+    const size_t p = pipe_layout(max_num_rows, K).total;
+    if (p > b) b = p;
+  }
+  return b;
 }
 
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route) {
@@ -1326,7 +1690,7 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
     const char* env = getenv("HPCTOPK_VARIANT");
     di.variant = env ? atoi(env) : kDefaultVariant;
-    if (di.variant != kFusedVariant && (di.variant < 0 || di.variant > kNumVariants)) di.variant = kDefaultVariant;
+    if (di.variant != kFusedVariant && di.variant != kPipeVariant && (di.variant < 0 || di.variant > kNumVariants)) di.variant = kDefaultVariant;
     if (cudaFuncSetAttribute(wsk::hpctopk_ws_kernel<wsk::kWsU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)wsk::ws_smem_bytes(HPCTOPK_MAX_K, true)) != cudaSuccess) {
       cudaGetLastError();
@@ -1353,6 +1717,32 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
         di.ctas_per_sm[sp][c] = n;
       }
     }
+    if (cudaFuncSetAttribute(kPassKernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(kRefineKernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    for (int c = 0; c < 3; ++c) {
+      for (int sp = 0; sp < 2; ++sp) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&di.pass_per_sm[sp][c], kPassKernel, kPassThreads,
+                                                          smem_bytes_for(class_cap_s(c), sp != 0)) != cudaSuccess ||
+            di.pass_per_sm[sp][c] < 1) {
+          cudaGetLastError();
+          return HPCTOPK_ERR_CUDA;
+        }
+      }
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&di.refine_per_sm[c], kRefineKernel, kRefineThreads,
+                                                        smem_bytes_for(0, false)) != cudaSuccess ||
+          di.refine_per_sm[c] < 1) {
+        cudaGetLastError();
+        return HPCTOPK_ERR_CUDA;
+      }
+    }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&di.boundary_per_sm, kBoundaryKernel, kBoundaryThreads,
+                                                      align_up(sizeof(Shared), 16)) != cudaSuccess || di.boundary_per_sm < 1) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
     di.ready = true;
   }
   const Variant& v = kVariants[variant_index(di.variant, split)];
@@ -1367,12 +1757,31 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);      // ceil(1.5 K / s)
   P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);      // ceil(1.75 K / s)
   P.split_enabled = split ? 1 : 0;
+  P.pipe_rec_off = P.pipe_cnt_off = P.pipe_cand_off = P.pipe_spill_off = 0;
   const size_t smem = smem_bytes_for(class_cap_s(cls), split);
   int grid = di.sm_count * di.ctas_per_sm[split ? 1 : 0][cls];
   if (grid > kMaxGrid) grid = kMaxGrid;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
-  if (di.variant == kFusedVariant) {
+  if (di.variant == kPipeVariant && num_rows <= kPipeRowsMax) {
+    const PipeLayout l = pipe_layout(num_rows, K);
+    P.pipe_rec_off = (int64_t)l.rec; P.pipe_cnt_off = (int64_t)l.cnt;
+    P.pipe_cand_off = (int64_t)l.cand; P.pipe_spill_off = (int64_t)l.spill;
+    int g1 = di.sm_count * di.boundary_per_sm;
+    if (g1 > num_rows) g1 = num_rows;
+    int g2 = di.sm_count * di.pass_per_sm[split ? 1 : 0][cls];
+    if (g2 > kMaxGrid) g2 = kMaxGrid;
+    int g3 = di.sm_count * di.refine_per_sm[cls];
+    if (g3 > kMaxGrid) g3 = kMaxGrid;
+    if (g3 > num_rows) g3 = num_rows;
+    kBoundaryKernel<<<g1, kBoundaryThreads, align_up(sizeof(Shared), 16), st>>>(P);
+    const char* stg = getenv("HPCTOPK_PIPE_STAGES");      // tuning aid: run only the first n kernels
+    const int stages = stg ? atoi(stg) : 3;
+    if (stages >= 2) kPassKernel<<<g2, kPassThreads, smem, st>>>(P);
+    Params R = P;
+    R.cap_s = 0;
+    if (stages >= 3) kRefineKernel<<<g3, kRefineThreads, smem_bytes_for(0, false), st>>>(R);
+  } else if (di.variant == kFusedVariant) {
     const size_t fsmem = wsf::ws_smem_bytes(K, split);
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wsf::hpctopk_ws_kernel<wsf::kWsU>, wsf::THREADS, fsmem) != cudaSuccess || per_sm < 1) {
@@ -1481,6 +1890,7 @@ extern "C" int hpctopk_select_static(const float* scores, const int32_t* row_sta
   P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);
   P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);
   P.split_enabled = 1;                                   // num_rows <= kStaticMaxRows <= kSplitRowsMax
+  P.pipe_rec_off = P.pipe_cnt_off = P.pipe_cand_off = P.pipe_spill_off = 0;
   int grid = sm_count[dev] * ctas_per_sm[dev][cls];
   if (grid > kStaticMaxGrid) grid = kStaticMaxGrid;
   if (static_layout_bytes((size_t)num_rows, (size_t)P.cap, (size_t)P.cap_s, (size_t)grid) > kStaticScratchBytes) return HPCTOPK_ERR_WORKSPACE;
