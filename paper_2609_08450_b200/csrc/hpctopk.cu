@@ -1578,6 +1578,8 @@ struct DeviceInfo {
   int pass_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // pipeline: pass kernel
   int refine_per_sm[3] = {0, 0, 0};                 // pipeline: refinement kernel
   int boundary_per_sm = 0;                          // pipeline: boundary kernel
+  bool pipe_split = false;                          // tuning: pipeline for split-mode calls too (HPCTOPK_PIPE_SPLIT)
+  int pipe_stages = 3;                              // tuning: run only the first n kernels (HPCTOPK_PIPE_STAGES)
 };
 DeviceInfo g_dev[64];
 
@@ -1688,6 +1690,8 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
     init_cut_table_kernel<<<kBins * 32 / 256, 256>>>();
     if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
+    di.pipe_split = getenv("HPCTOPK_PIPE_SPLIT") != nullptr;
+    if (const char* stg = getenv("HPCTOPK_PIPE_STAGES")) di.pipe_stages = atoi(stg);
     const char* env = getenv("HPCTOPK_VARIANT");
     di.variant = env ? atoi(env) : kDefaultVariant;
     if (di.variant != kFusedVariant && di.variant != kPipeVariant && (di.variant < 0 || di.variant > kNumVariants)) di.variant = kDefaultVariant;
@@ -1763,7 +1767,8 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   if (grid > kMaxGrid) grid = kMaxGrid;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
-  if (di.variant == kPipeVariant && num_rows <= kPipeRowsMax) {
+  // Calls of few rows (split mode) are latency-bound: one launch and on-chip tails serve them better.
+  if (di.variant == kPipeVariant && num_rows <= kPipeRowsMax && (!split || di.pipe_split)) {
     const PipeLayout l = pipe_layout(num_rows, K);
     P.pipe_rec_off = (int64_t)l.rec; P.pipe_cnt_off = (int64_t)l.cnt;
     P.pipe_cand_off = (int64_t)l.cand; P.pipe_spill_off = (int64_t)l.spill;
@@ -1775,8 +1780,7 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     if (g3 > kMaxGrid) g3 = kMaxGrid;
     if (g3 > num_rows) g3 = num_rows;
     kBoundaryKernel<<<g1, kBoundaryThreads, align_up(sizeof(Shared), 16), st>>>(P);
-    const char* stg = getenv("HPCTOPK_PIPE_STAGES");      // tuning aid: run only the first n kernels
-    const int stages = stg ? atoi(stg) : 3;
+    const int stages = di.pipe_stages;
     if (stages >= 2) kPassKernel<<<g2, kPassThreads, smem, st>>>(P);
     Params R = P;
     R.cap_s = 0;

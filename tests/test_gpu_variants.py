@@ -1,7 +1,9 @@
-"""The alternative kernels (warp-specialised, fused single-role) against the oracle.
+"""The alternative kernels against the oracle: warp-specialised (0), fused single-role (100),
+another launch shape (2), the single kernel for every call shape (4), and the three-kernel
+pipeline for split-mode calls too (default variant with HPCTOPK_PIPE_SPLIT set).
 
-The variant is chosen once per process from the HPCTOPK_VARIANT environment variable, so each
-one runs in a child process."""
+The variant is chosen once per process from environment variables, so each one runs in a child
+process."""
 import os
 import subprocess
 import sys
@@ -12,9 +14,11 @@ pytestmark = pytest.mark.gpu
 HERE = os.path.dirname(os.path.abspath(__file__))
 
 
-@pytest.mark.parametrize("variant", ["0", "100", "2"])
+@pytest.mark.parametrize("variant", ["0", "100", "2", "4", "200+split"])
 def test_variant_matches_oracle(variant):
-    env = dict(os.environ, HPCTOPK_VARIANT=variant)
+    env = dict(os.environ, HPCTOPK_VARIANT=variant.split("+")[0])
+    if variant.endswith("+split"):
+        env["HPCTOPK_PIPE_SPLIT"] = "1"
     out = subprocess.run([sys.executable, os.path.join(HERE, "variant_check.py")], env=env, capture_output=True,
                          text=True, timeout=600)
     assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
