@@ -91,6 +91,7 @@ struct Params {
   // Three-kernel pipeline only (zero otherwise): workspace offsets of the per-row boundary
   // records, the per-row admitted counts, the per-row candidate ranges and the overflow slices.
   int64_t pipe_rec_off, pipe_cnt_off, pipe_cand_off, pipe_spill_off;
+  int32_t row_begin, row_end;   // the rows this launch of a pipeline kernel covers
 };
 
 // What the boundary kernel leaves for a row and the other two kernels read.
@@ -282,22 +283,6 @@ __device__ __forceinline__ void w_clear_hist(uint32_t* hist, int lane) {
 #pragma unroll
   for (int b = 0; b < 16; ++b) hv[b * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
 }
-// Three bin -> cutoff searches advanced together (see cutoff_of_bin): 32 probes per step each.
-__device__ __forceinline__ void w_cutoffs3(const int (&tau)[3], uint32_t (&cut)[3], int lane) {
-  uint32_t lo[3] = {0u, 0u, 0u};
-#pragma unroll 1
-  for (int b = 27; b >= -3; b -= 5) {
-    const int sh = b < 0 ? 0 : b;
-    const uint32_t nprobe = b < 0 ? 3u : 31u;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-      const uint64_t probe = (uint64_t)lo[k] + ((uint64_t)(lane + 1) << sh);
-      const bool ok = (uint32_t)lane < nprobe && probe <= 0xFFFFFFFFull && coarse_bin_of_kd((uint32_t)probe) <= tau[k];
-      lo[k] += (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, ok)) << sh;
-    }
-  }
-  cut[0] = lo[0]; cut[1] = lo[1]; cut[2] = lo[2];
-}
 
 // ---------------------------------------------------------------- block primitives
 template <int THREADS>
@@ -422,13 +407,6 @@ struct Admit {
     bound = (int32_t)(cu ^ flip);
   }
   __device__ __forceinline__ bool operator()(uint32_t u) const { return (int32_t)(u ^ flip) >= bound; }
-  __device__ __forceinline__ bool negative() const { return flip != 0u; }
-  template <int MODE>
-  __device__ __forceinline__ bool test(uint32_t u) const {
-    if (MODE == 1) return (int32_t)u >= bound;                       // cutoff positive
-    if (MODE == 2) return u <= ((uint32_t)bound ^ 0x7FFFFFFFu);      // cutoff negative
-    return (*this)(u);
-  }
 };
 
 // Where admitted scores go: shared memory first, then this CTA's global overflow slice.
@@ -446,18 +424,8 @@ __device__ __forceinline__ CandCtx cand_ctx(const Params& P) {
   c.spill = reinterpret_cast<uint2*>(P.ws + spill_off) + (size_t)blockIdx.x * (size_t)(P.cap - P.cap_s);
   return c;
 }
-#ifdef HPCTOPK_RAW
-constexpr bool kRawEntries = true;     // entries hold the raw bits; the key is formed when an entry is read
-#else
-constexpr bool kRawEntries = false;
-#endif
-__device__ __forceinline__ uint2 cand_raw(const CandCtx& c, uint32_t i) {
-  return i < c.cap_s ? CAND()[i] : __ldcg(c.spill + (i - c.cap_s));
-}
 __device__ __forceinline__ uint2 cand_load(const CandCtx& c, uint32_t i) {   // (kd, idx)
-  uint2 e = cand_raw(c, i);
-  if (kRawEntries) e.x = kd_of_bits(e.x);
-  return e;
+  return i < c.cap_s ? CAND()[i] : __ldcg(c.spill + (i - c.cap_s));
 }
 __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v) {
   if (i < c.cap_s) CAND()[i] = v; else c.spill[i - c.cap_s] = v;
@@ -475,7 +443,7 @@ __device__ __forceinline__ void cand_store(const CandCtx& c, uint32_t i, uint2 v
 // form makes the whole warp wait at its votes and shuffles.)
 __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const CandCtx& c) {
   Shared& sh = SH();
-  const uint32_t kd = kRawEntries ? u : kd_of_bits(u);
+  const uint32_t kd = kd_of_bits(u);
   const uint32_t pos = atomicAdd(&sh.cand_count, 1u);
   if (pos < c.cap_s) CAND()[pos] = make_uint2(kd, idx);
   else if (pos < c.cap) c.spill[pos - c.cap_s] = make_uint2(kd, idx);
@@ -487,14 +455,14 @@ __device__ __forceinline__ void append_candidate(uint32_t u, uint32_t idx, const
 //   BAND = true : admit cut_lo < kd <= cut_hi.   (the band of Eq. "rescue-band")
 // Admitted scores are rare (about 1.5 K / L of the row), so the loop spends one compare and one
 // branch per score and leaves everything else to the taken branch.
-template <int THREADS, int U, bool BAND, int MODE>
-__device__ __forceinline__ void scan_body(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
+template <int THREADS, int U, bool BAND>
+__device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
                                              uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
   const int tid = threadIdx.x;
   if (e1 <= e0) return;
   const Admit in_hi(cut_hi);
   const Admit in_lo(cut_lo);                 // BAND: scores admitted by tau_0 are already held
-  auto admit = [&](uint32_t u) -> bool { return BAND ? (in_hi(u) && !in_lo(u)) : in_hi.template test<MODE>(u); };
+  auto admit = [&](uint32_t u) -> bool { return BAND ? (in_hi(u) && !in_lo(u)) : in_hi(u); };
   int64_t b0 = (e0 + 3) & ~(int64_t)3;       // first 16-byte aligned element
   int64_t b1 = e1 & ~(int64_t)3;             // end of the last whole vector
   if (b0 > b1) { b0 = e1; b1 = e1; }         // range holds no whole vector
@@ -556,30 +524,6 @@ __device__ __forceinline__ void scan_body(const float* __restrict__ scores, int6
   for (int64_t v = nfull * TILE + tid; v < nvec; v += THREADS)
     classify(__ldcs(vp + v), idx0 + (uint32_t)(v << 2));
 }
-
-#ifndef HPCTOPK_SIGNSPEC
-template <int THREADS, int U, bool BAND>
-__device__ __noinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
-                                        uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
-  scan_body<THREADS, U, BAND, 0>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
-}
-#else
-template <int THREADS, int U, bool BAND, int MODE>
-__device__ __noinline__ void scan_range_m(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
-                                          uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
-  scan_body<THREADS, U, BAND, MODE>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
-}
-template <int THREADS, int U, bool BAND>
-__device__ __forceinline__ void scan_range(const float* __restrict__ scores, int64_t g0, int64_t e0, int64_t e1,
-                                           uint32_t cut_lo, uint32_t cut_hi, const CandCtx cc) {
-  if (!BAND) {                               // one compare per score, by the sign of the cutoff
-    if (Admit(cut_hi).negative()) scan_range_m<THREADS, U, false, 2>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
-    else scan_range_m<THREADS, U, false, 1>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
-    return;
-  }
-  scan_range_m<THREADS, U, BAND, 0>(scores, g0, e0, e1, cut_lo, cut_hi, cc);
-}
-#endif
 
 // ---------------------------------------------------------------- element sources for selection
 // A source visits every element once per pass, calling f(valid, kd, idx) with a block-uniform
@@ -748,7 +692,7 @@ __device__ void record_row(const Params& P, int row, int route, int tau, uint32_
 }
 
 // Phase 1 (Section 4.2): sample view -> coarse histogram -> tau_0, tau_1 -> cutoffs in sh.cutd.
-// A third, tighter bin tau_hi at half the rank K (sample rank ceil(K / 2s)) brackets the K-th
+// A third, tighter bin tau_hi at a quarter of the rank K (sample rank ceil(K / 4s)) brackets the K-th
 // score from above; its cutoff sizes the refinement digit of select_adaptive.
 // Returns false when the view cannot support the requested sample ranks.
 template <int THREADS, bool BLOCK_SEARCH = false>
@@ -792,7 +736,7 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   __syncthreads();
   DSTAMP(6, ts);
   {
-    int q_hi = (P.K + 2 * s - 1) / (2 * s);
+    int q_hi = (P.K + 4 * s - 1) / (4 * s);                           // bracket: sample rank ceil(K/4s)
     if (q_hi < 1) q_hi = 1;
     const uint32_t q2 = (uint32_t)((3 * P.K + s - 1) / s);             // second band: sample rank ceil(3K/s)
     const uint32_t quota[4] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi, q2};
@@ -852,6 +796,7 @@ template <int THREADS, bool BLOCK_SEARCH = false, bool COUNT0 = false>
 __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint32_t K, uint32_t cut_base, uint32_t cut_hi,
                                              int32_t* out_idx, float* out_val, uint32_t cut_count = 0u) {
   Shared& sh = SH();
+  constexpr int W = THREADS <= 128 ? 8 : 4;      // entries per thread and batch (independent loads in flight)
   const int tid = threadIdx.x, lane = tid & 31;
   const uint32_t span = cut_base > cut_hi ? cut_base - cut_hi : 0u;
   int shv = 0;
@@ -868,18 +813,18 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
   __syncthreads();
   DSTAMP(0, ts);
   uint32_t n0 = 0;                               // COUNT0: entries with kd <= cut_count, added to sh.count0
-  for (uint32_t i0 = 0; i0 < C; i0 += 4 * THREADS) {
-    uint2 c[4];
-    bool v[4];
+  for (uint32_t i0 = 0; i0 < C; i0 += W * THREADS) {
+    uint2 c[W];
+    bool v[W];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < W; ++k) {
       const uint32_t i = i0 + k * THREADS + tid;
       c[k] = i < C ? cand_load(cc, i) : make_uint2(0xFFFFFFFFu, 0u);
       v[k] = i < C && c[k].x <= cut_base;       // a split row's buffer also holds the band beyond tau_0
       if (COUNT0) n0 += (i < C && c[k].x <= cut_count) ? 1u : 0u;
     }
 #pragma unroll
-    for (int k = 0; k < 4; ++k) if (v[k]) atomicAdd(&sh.hist[digit(c[k].x)], 1u);
+    for (int k = 0; k < W; ++k) if (v[k]) atomicAdd(&sh.hist[digit(c[k].x)], 1u);
   }
   if (COUNT0) {
     n0 = __reduce_add_sync(0xFFFFFFFFu, n0);
@@ -906,12 +851,12 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
   const uint32_t k_rem = K - below;             // to take from the boundary bin
   uint2* const list = reinterpret_cast<uint2*>(sh.hist);
   __syncthreads();                              // the histogram's memory becomes the boundary list
-  for (uint32_t i0 = 0; i0 < C; i0 += 4 * THREADS) {
-    uint2 c[4];
-    uint32_t dg[4];
+  for (uint32_t i0 = 0; i0 < C; i0 += W * THREADS) {
+    uint2 c[W];
+    uint32_t dg[W];
     uint32_t cnt = 0;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < W; ++k) {
       const uint32_t i = i0 + k * THREADS + tid;
       c[k] = i < C ? cand_load(cc, i) : make_uint2(0xFFFFFFFFu, 0u);
       dg[k] = (i < C && c[k].x <= cut_base) ? digit(c[k].x) : 0xFFFFFFFFu;
@@ -924,7 +869,7 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
     base = __shfl_sync(0xFFFFFFFFu, base, 31);
     uint32_t pos = base + incl - cnt;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < W; ++k) {
       if (dg[k] < (uint32_t)b) {
         if (pos < K) { out_idx[pos] = (int32_t)c[k].y; if (out_val) out_val[pos] = __uint_as_float(bits_of_kd(c[k].x)); }
         ++pos;
@@ -1027,9 +972,8 @@ __device__ void finish_sampled_row(const Params& P, const CandCtx cc, int row, i
 
 // A row owned by one CTA from Phase 1 to the output commit.
 template <int THREADS, int U>
-__device__ void process_row(const Params& P, int row) {
+__device__ void process_row(const Params& P, int row, const CandCtx cc) {
   Shared& sh = SH();
-  const CandCtx cc = cand_ctx(P);
   const int64_t g0 = P.row_starts[row];
   int64_t L = P.row_lengths[row];
   if (L < 0) L = 0;
@@ -1129,7 +1073,7 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   __syncthreads();
   const uint32_t base = sh.bcast0;
   if (base + Cp <= cap) {
-    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gcand[base + i] = cand_raw(cc, i);
+    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gcand[base + i] = cand_load(cc, i);
   }
   __threadfence();
   __syncthreads();
@@ -1274,10 +1218,10 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
       while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (seg_base[mid] <= task) lo = mid; else hi = mid - 1; }
       const int row = lo;
       const int nseg = (int)(seg_base[row + 1] - seg_base[row]);
-      if (nseg <= 1) process_row<THREADS, U>(P, row);
+      if (nseg <= 1) process_row<THREADS, U>(P, row, cand_ctx(P));
       else process_segment<THREADS, U>(P, row, (int)(task - seg_base[row]), nseg);
     } else {
-      process_row<THREADS, U>(P, row_of_task(P, task));
+      process_row<THREADS, U>(P, row_of_task(P, task), cand_ctx(P));
     }
     __syncthreads();
     const uint32_t claimed = (uint32_t)sh.claim;
@@ -1315,7 +1259,7 @@ __global__ void __launch_bounds__(THREADS) pipe_boundary_kernel(const Params P) 
   Shared& sh = SH();
   stats_clear();
   __syncthreads();
-  for (int row = blockIdx.x; row < P.num_rows; row += gridDim.x) {
+  for (int row = P.row_begin + blockIdx.x; row < P.row_end; row += gridDim.x) {
     const int64_t g0 = P.row_starts[row];
     const int64_t L = P.row_lengths[row];
     int tau_pack = -1;
@@ -1333,11 +1277,13 @@ __global__ void __launch_bounds__(THREADS) pipe_boundary_kernel(const Params P) 
   }
 }
 
-// One task of the pass kernel: elements [e0, e1) of a sampled row.
+// The pass kernel's work on one row.
 template <int THREADS, int U>
-__device__ void pipe_pass_task(const Params& P, int row, int seg, int nseg) {
+__device__ void pipe_pass_task(const Params& P, int row) {
   Shared& sh = SH();
-  const CandCtx cc = cand_ctx(P);
+  // entries beyond the on-chip part go straight to their place in the row's global range
+  CandCtx cc;
+  cc.cap_s = (uint32_t)P.cap_s; cc.cap = (uint32_t)P.cap; cc.spill = pipe_cand(P, row) + P.cap_s;
   const int64_t g0 = P.row_starts[row];
   const int64_t L = P.row_lengths[row];
   if (L <= (int64_t)P.cap) return;                       // short and direct rows: refinement kernel
@@ -1347,25 +1293,15 @@ __device__ void pipe_pass_task(const Params& P, int row, int seg, int nseg) {
   if (r1.y == 0u) return;                                // unusable view: refinement kernel recovers
   const uint32_t cut1 = r0.y, cap = (uint32_t)P.cap;
   const int64_t g1 = g0 + L;
-  int64_t e0 = g0, e1 = g1;
-  if (nseg > 1) {                                        // contiguous, 16-byte aligned partition
-    const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
-    const int64_t per = (vb - va + nseg - 1) / nseg;
-    e0 = (va + (int64_t)seg * per) << 2;
-    e1 = (va + (int64_t)(seg + 1) * per) << 2;
-    if (e0 < g0) e0 = g0;
-    if (e1 > g1) e1 = g1;
-    if (e1 < e0) e1 = e0;
-  }
   __syncthreads();
   if (threadIdx.x == 0) sh.cand_count = 0;
   __syncthreads();
-  scan_range<THREADS, U, false>(P.scores, g0, e0, e1, 0u, cut1, cc);
+  scan_range<THREADS, U, false>(P.scores, g0, g0, g1, 0u, cut1, cc);
   __syncthreads();
   uint32_t Cp = sh.cand_count;
   uint32_t flag = 0u;
-  uint64_t scanned = (uint64_t)(e1 - e0);
-  if (nseg == 1 && Cp < (uint32_t)P.K && r0.w > cut1) {
+  uint64_t scanned = (uint64_t)L;
+  if (Cp < (uint32_t)P.K && r0.w > cut1) {
     // Underfilled row owned by this CTA: append the second band (tau_1, tau_2] here, where the
     // row has just passed through the L2 and 16 warps stream it, and tell the refinement kernel.
     __syncthreads();
@@ -1376,56 +1312,28 @@ __device__ void pipe_pass_task(const Params& P, int row, int seg, int nseg) {
     scanned += (uint64_t)L;
   }
   if (threadIdx.x == 0) {
-    sh.bcast0 = atomicAdd(&pipe_cnt(P)[row], Cp | flag) & ~kBand2Flag;
-    hpctopk_stats* st = stats_of(P.ws);
-    add64(&st->elements_scanned, scanned);
-    if (nseg > 1 && seg == 0) add64(&st->rows_split, 1);
+    pipe_cnt(P)[row] = Cp | flag;
+    add64(&stats_of(P.ws)->elements_scanned, scanned);
   }
-  __syncthreads();
-  const uint32_t base = sh.bcast0;
-  if (Cp <= cap && base + Cp <= cap) {                   // otherwise the row total exceeds the capacity anyway
-    uint2* gc = pipe_cand(P, row) + base;
-    for (uint32_t i = threadIdx.x; i < Cp; i += THREADS) gc[i] = cand_raw(cc, i);
+  if (Cp <= cap) {                                       // otherwise the refinement kernel recovers the row
+    uint2* gc = pipe_cand(P, row);
+    const uint32_t on_chip = Cp < cc.cap_s ? Cp : cc.cap_s;
+    for (uint32_t i = threadIdx.x; i < on_chip; i += THREADS) gc[i] = CAND()[i];
   }
 }
 
+// One CTA per row, longest rows (highest row numbers of a causal batch) first; the hardware
+// hands out CTAs as SM resources free up, across the launches of consecutive row chunks.
 template <int THREADS, int U, int MINB>
 __global__ void __launch_bounds__(THREADS, MINB) pipe_pass_kernel(const Params P) {
-  Shared& sh = SH();
-  uint32_t* const seg_base = reinterpret_cast<uint32_t*>(CAND() + P.cap_s);   // [kSplitRowsMax + 1], only when splitting
-  uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl);
-  const int tid = threadIdx.x;
   stats_clear();
   __syncthreads();
-  uint32_t total_tasks = (uint32_t)P.num_rows;
-  if (P.split_enabled) total_tasks = build_task_table<THREADS>(P, seg_base);
-  uint32_t task = blockIdx.x;
-  uint32_t next = blockIdx.x + gridDim.x;
-  while (task < total_tasks) {
-    if (tid == 0) sh.claim = (int32_t)(2u * gridDim.x + atomicAdd(task_counter, 1u));
-#ifdef HPCTOPK_PASS_PREFETCH
-    if (!P.split_enabled && next < total_tasks) {
-      const int nrow = row_of_task(P, next);
-      const int64_t ng0 = P.row_starts[nrow], nL = P.row_lengths[nrow];
-      if (nL > P.cap) prefetch_head<THREADS>(P, ng0, ng0 + nL);
-    }
-#endif
-    if (P.split_enabled) {
-      int lo = 0, hi = P.num_rows - 1;
-      while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (seg_base[mid] <= task) lo = mid; else hi = mid - 1; }
-      pipe_pass_task<THREADS, U>(P, lo, (int)(task - seg_base[lo]), (int)(seg_base[lo + 1] - seg_base[lo]));
-    } else {
-      pipe_pass_task<THREADS, U>(P, row_of_task(P, task), 0, 1);
-    }
-    __syncthreads();
-    const uint32_t claimed = (uint32_t)sh.claim;
-    if (tid == 0) add64(&stats_of(P.ws)->tasks, 1);
-    __syncthreads();
-    task = next;
-    next = claimed;
-  }
+  pipe_pass_task<THREADS, U>(P, P.row_end - 1 - (int)blockIdx.x);
   __syncthreads();
-  if (tid == 0) stats_flush(P.ws);
+  if (threadIdx.x == 0) {
+    add64(&stats_of(P.ws)->tasks, 1);
+    stats_flush(P.ws);
+  }
 }
 
 // The refinement kernel keeps no candidates on chip: it reads a row's admitted tail from its
@@ -1436,32 +1344,20 @@ __global__ void __launch_bounds__(THREADS, MINB) pipe_pass_kernel(const Params P
 template <int THREADS, int U, int MINB>
 __global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params P) {
   Shared& sh = SH();
-  uint32_t* task_counter = reinterpret_cast<uint32_t*>(P.ws + kOffCtrl) + 1;
   const int tid = threadIdx.x;
   const uint32_t cap = (uint32_t)P.cap, K = (uint32_t)P.K;
   stats_clear();
   __syncthreads();
-  long long t_life = tick();
-#if HPCTOPK_TIMERS
-  unsigned long long gt0; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0));
-#endif
-  // Every row is claimed from the device counter, the first one too: a CTA that becomes resident
-  // late (the grid may exceed what the SMs hold at once) then finds the rows already taken
-  // instead of sitting on a statically assigned one.
-  if (tid == 0) sh.claim = (int32_t)atomicAdd(task_counter, 1u);
-  __syncthreads();
-  uint32_t task = (uint32_t)sh.claim;
-  __syncthreads();
-  while (task < (uint32_t)P.num_rows) {
-    long long ts = tick();
-    if (tid == 0) sh.claim = (int32_t)atomicAdd(task_counter, 1u);
-    const int row = row_of_task(P, task);
+  {
+    const int row = P.row_end - 1 - (int)blockIdx.x;
     const int64_t g0 = P.row_starts[row];
     const int64_t L = P.row_lengths[row];
     const RowRec* rec = pipe_rec(P) + row;
     const bool sampled = L > (int64_t)cap && __ldg(&rec->usable) != 0u;
     if (!sampled) {
-      process_row<THREADS, U>(P, row);                   // short, direct, or recovery of an unusable view
+      CandCtx rc;                                        // staging area: the row's own global range
+      rc.cap_s = 0u; rc.cap = cap; rc.spill = pipe_cand(P, row);
+      process_row<THREADS, U>(P, row, rc);               // short, direct, or recovery of an unusable view
     } else {
       __syncthreads();
       if (tid < 4) sh.cutd[tid] = __ldg(&rec->cutd[tid]);
@@ -1503,16 +1399,8 @@ __global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params
                    4ull * (uint64_t)L, sampled_n, (uint64_t)L);
       }
     }
-    __syncthreads();
-    const uint32_t claimed = (uint32_t)sh.claim;
-    __syncthreads();
-    task = claimed;
   }
   __syncthreads();
-  DSTAMP(5, t_life);
-#if HPCTOPK_TIMERS
-  if (tid == 0) { unsigned long long gt1; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1)); atomicAdd(reinterpret_cast<unsigned long long*>(&stats_of(nullptr)->cycles_detail[7]), gt1 - gt0); atomicMax(reinterpret_cast<unsigned long long*>(&stats_of(nullptr)->candidates_max), gt1 - gt0); }
-#endif
   if (tid == 0) stats_flush(P.ws);
 }
 
@@ -1575,10 +1463,7 @@ struct DeviceInfo {
   int sm_count = 0;
   int variant = 0;      // 0: warp-specialised kernel; v >= 1: single-role kernel kVariants[v - 1]
   int ctas_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // [split][capacity class]
-  int pass_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // pipeline: pass kernel
-  int refine_per_sm[3] = {0, 0, 0};                 // pipeline: refinement kernel
   int boundary_per_sm = 0;                          // pipeline: boundary kernel
-  bool pipe_split = false;                          // tuning: pipeline for split-mode calls too (HPCTOPK_PIPE_SPLIT)
   int pipe_stages = 3;                              // tuning: run only the first n kernels (HPCTOPK_PIPE_STAGES)
 };
 DeviceInfo g_dev[64];
@@ -1602,19 +1487,17 @@ int cap_class(int K) { return K <= 1024 ? 0 : (K <= 2048 ? 1 : 2); }
 int class_cap_s(int cls) { return smem_capacity_for(cls == 0 ? 1024 : (cls == 1 ? 2048 : HPCTOPK_MAX_K)); }
 
 // Workspace layout of the pipeline: the common head (control block, counters, row records of
-// hpctopk_read_row_info), then boundary records, admitted counts, one candidate range of
-// `capacity` entries per row, and the overflow slices.
-struct PipeLayout { size_t rec, cnt, cand, spill, total; };
+// hpctopk_read_row_info), then boundary records, admitted counts and one candidate range of
+// `capacity` entries per row (a pass CTA writes what exceeds its shared memory straight into
+// that range, and the refinement kernel stages nothing on chip, so there are no overflow slices).
+struct PipeLayout { size_t rec, cnt, cand, total; };
 PipeLayout pipe_layout(int rows, int K) {
   const size_t cap = (size_t)capacity_for(K);
-  const int cap_s_cls = class_cap_s(cap_class(K));
-  const size_t cap_s = (size_t)cap_s_cls < cap ? (size_t)cap_s_cls : cap;
   PipeLayout l;
   l.rec = align_up(kOffRowInfo + (size_t)rows * sizeof(hpctopk_row_info), 256);
   l.cnt = align_up(l.rec + (size_t)rows * sizeof(RowRec), 256);
   l.cand = align_up(l.cnt + (size_t)rows * sizeof(uint32_t), 256);
-  l.spill = l.cand + (size_t)rows * cap * 8;
-  l.total = align_up(l.spill + (size_t)kMaxGrid * cap * 8, 256);   // the refinement kernel stages nothing on chip
+  l.total = align_up(l.cand + (size_t)rows * cap * 8, 256);
   return l;
 }
 
@@ -1690,7 +1573,6 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
     init_cut_table_kernel<<<kBins * 32 / 256, 256>>>();
     if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
-    di.pipe_split = getenv("HPCTOPK_PIPE_SPLIT") != nullptr;
     if (const char* stg = getenv("HPCTOPK_PIPE_STAGES")) di.pipe_stages = atoi(stg);
     const char* env = getenv("HPCTOPK_VARIANT");
     di.variant = env ? atoi(env) : kDefaultVariant;
@@ -1726,22 +1608,6 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
       cudaGetLastError();
       return HPCTOPK_ERR_CUDA;
     }
-    for (int c = 0; c < 3; ++c) {
-      for (int sp = 0; sp < 2; ++sp) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&di.pass_per_sm[sp][c], kPassKernel, kPassThreads,
-                                                          smem_bytes_for(class_cap_s(c), sp != 0)) != cudaSuccess ||
-            di.pass_per_sm[sp][c] < 1) {
-          cudaGetLastError();
-          return HPCTOPK_ERR_CUDA;
-        }
-      }
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&di.refine_per_sm[c], kRefineKernel, kRefineThreads,
-                                                        smem_bytes_for(0, false)) != cudaSuccess ||
-          di.refine_per_sm[c] < 1) {
-        cudaGetLastError();
-        return HPCTOPK_ERR_CUDA;
-      }
-    }
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&di.boundary_per_sm, kBoundaryKernel, kBoundaryThreads,
                                                       align_up(sizeof(Shared), 16)) != cudaSuccess || di.boundary_per_sm < 1) {
       cudaGetLastError();
@@ -1768,23 +1634,25 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
   // Calls of few rows (split mode) are latency-bound: one launch and on-chip tails serve them better.
-  if (di.variant == kPipeVariant && num_rows <= kPipeRowsMax && (!split || di.pipe_split)) {
+  if (di.variant == kPipeVariant && num_rows <= kPipeRowsMax && !split) {
     const PipeLayout l = pipe_layout(num_rows, K);
     P.pipe_rec_off = (int64_t)l.rec; P.pipe_cnt_off = (int64_t)l.cnt;
-    P.pipe_cand_off = (int64_t)l.cand; P.pipe_spill_off = (int64_t)l.spill;
+    P.pipe_cand_off = (int64_t)l.cand;
+    // Three launches on the caller's stream.  (Cutting the rows into chunks and overlapping the
+    // boundary and refinement kernels of neighbouring chunks with the pass kernel on extra streams
+    // was measured: no gain, the streaming CTAs leave no room on the SMs until they exit, and
+    // limiting them to two per SM costs the pass kernel more than the overlap returns.)
+    P.row_begin = 0;
+    P.row_end = num_rows;
+    const size_t smem_pass = smem_bytes_for(class_cap_s(cls), false);
+    const size_t smem_small = smem_bytes_for(0, false);
     int g1 = di.sm_count * di.boundary_per_sm;
     if (g1 > num_rows) g1 = num_rows;
-    int g2 = di.sm_count * di.pass_per_sm[split ? 1 : 0][cls];
-    if (g2 > kMaxGrid) g2 = kMaxGrid;
-    int g3 = di.sm_count * di.refine_per_sm[cls];
-    if (g3 > kMaxGrid) g3 = kMaxGrid;
-    if (g3 > num_rows) g3 = num_rows;
-    kBoundaryKernel<<<g1, kBoundaryThreads, align_up(sizeof(Shared), 16), st>>>(P);
-    const int stages = di.pipe_stages;
-    if (stages >= 2) kPassKernel<<<g2, kPassThreads, smem, st>>>(P);
+    kBoundaryKernel<<<g1, kBoundaryThreads, smem_small, st>>>(P);
+    if (di.pipe_stages >= 2) kPassKernel<<<num_rows, kPassThreads, smem_pass, st>>>(P);
     Params R = P;
     R.cap_s = 0;
-    if (stages >= 3) kRefineKernel<<<g3, kRefineThreads, smem_bytes_for(0, false), st>>>(R);
+    if (di.pipe_stages >= 3) kRefineKernel<<<num_rows, kRefineThreads, smem_small, st>>>(R);
   } else if (di.variant == kFusedVariant) {
     const size_t fsmem = wsf::ws_smem_bytes(K, split);
     int per_sm = 0;

@@ -1,8 +1,8 @@
 """The alternative kernels against the oracle: warp-specialised (0), fused single-role (100),
-another launch shape (2), the single kernel for every call shape (4), and the three-kernel
-pipeline for split-mode calls too (default variant with HPCTOPK_PIPE_SPLIT set).
+another launch shape (2), and the single kernel for every call shape (4; the default takes the
+three-kernel pipeline for calls of more than 512 rows).
 
-The variant is chosen once per process from environment variables, so each one runs in a child
+The variant is chosen once per process from an environment variable, so each one runs in a child
 process."""
 import os
 import subprocess
@@ -14,11 +14,9 @@ pytestmark = pytest.mark.gpu
 HERE = os.path.dirname(os.path.abspath(__file__))
 
 
-@pytest.mark.parametrize("variant", ["0", "100", "2", "4", "200+split"])
+@pytest.mark.parametrize("variant", ["0", "100", "2", "4"])
 def test_variant_matches_oracle(variant):
-    env = dict(os.environ, HPCTOPK_VARIANT=variant.split("+")[0])
-    if variant.endswith("+split"):
-        env["HPCTOPK_PIPE_SPLIT"] = "1"
+    env = dict(os.environ, HPCTOPK_VARIANT=variant)
     out = subprocess.run([sys.executable, os.path.join(HERE, "variant_check.py")], env=env, capture_output=True,
                          text=True, timeout=600)
     assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
