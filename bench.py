@@ -27,10 +27,12 @@ import numpy as np
 import torch
 
 K = 2048
-# DRAM bytes per score element of the dominant kernel, from the ncu capture summarised in
-# profiles/hpctopk_kernel_config3_small.md (dram__bytes_read.sum + dram__bytes_write.sum over
-# the valid elements of the captured launch; traffic grows in proportion to the elements).
-NCU_DRAM_BYTES_PER_ELEMENT = 4.83
+# DRAM bytes per score element of the dominant kernel (pipe_pass_kernel), from the ncu capture
+# summarised in profiles/pipeline_config3_full.md (dram__bytes_read.sum + dram__bytes_write.sum of
+# one launch on the full workload, single-pass metrics, over its valid elements).
+NCU_DRAM_BYTES_PER_ELEMENT = 4.17
+# the single kernel (calls of at most 512 rows), from profiles/hpctopk_kernel_config3_small.md
+NCU_DRAM_BYTES_PER_ELEMENT_SINGLE = 4.83
 
 
 def load_peaks():
@@ -218,6 +220,8 @@ def main():
     barrier()
     starts_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    B.hpctopk_stage_timing(True)          # CUDA events around the dominant kernel of every call
+    B.hpctopk_read_stage_timing()
     with ClockSampler(local_rank) as clocks:
         barrier()
         for i in range(args.steps):
@@ -227,6 +231,8 @@ def main():
             step()
             ends_ev[i].record(stream)
         barrier()
+    dom_ms, dom_calls = B.hpctopk_read_stage_timing()
+    B.hpctopk_stage_timing(False)
     ms = [s.elapsed_time(e) for s, e in zip(starts_ev, ends_ev)]
     total_ms = sharding.max_over_ranks(sum(ms), dev)
     all_elems = sharding.sum_over_ranks(n_elem, dev)
@@ -267,8 +273,13 @@ def main():
         peak, peak_kind = load_peaks()
         value = all_elems * args.steps / (total_ms * 1e-3)
         local_ms = float(np.mean(ms))
-        achieved = 4.0 * n_elem / (local_ms * 1e-3) / 1e9        # GB/s of algorithmic score bytes
-        traffic = None if NCU_DRAM_BYTES_PER_ELEMENT is None else NCU_DRAM_BYTES_PER_ELEMENT * n_elem
+        # dominant kernel: the pass kernel of a three-kernel call (every score is read there, once),
+        # the one kernel otherwise; its launches were timed inside the region above
+        kernels = B.hpctopk_kernels_per_call(M)
+        dom_ms_per_launch = dom_ms / max(dom_calls, 1)
+        achieved = 4.0 * n_elem / (dom_ms_per_launch * 1e-3) / 1e9   # GB/s of algorithmic score bytes
+        achieved_call = 4.0 * n_elem / (local_ms * 1e-3) / 1e9       # the same over the whole call
+        traffic = (NCU_DRAM_BYTES_PER_ELEMENT if kernels == 3 else NCU_DRAM_BYTES_PER_ELEMENT_SINGLE) * n_elem
         line = {
             "metric": "score elements/s, exact Top-K K=2048", "value": value, "unit": "score elements/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
@@ -279,11 +290,15 @@ def main():
                        "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps (512 MB write)"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                         "kernel": "pipe_pass_kernel<512,2,3>" if kernels == 3 else "hpctopk_kernel",
+                         "kernel_ms_per_launch": dom_ms_per_launch, "kernel_launches_timed": dom_calls,
+                         "whole_call": {"achieved": achieved_call, "frac": achieved_call / peak,
+                                        "kernels_per_call": kernels},
                          "frac_of_nominal_8TBs": achieved / 8000.0,
                          "algorithmic_bytes": "4 bytes per valid score (one complete-row read)"},
             "e2e": {"value": all_elems * args.e2e_steps / (e2e_ms * 1e-3), "unit": "score elements/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": args.steps,
+            "gpu_launches": args.steps * B.hpctopk_kernels_per_call(M),
             "clocks": clocks.summary(),
             "routes": {k: v for k, v in stats.items() if k.startswith("rows_")},
             "row_equivalent_reads": (stats["elements_scanned"] + stats["elements_sampled"]) / max(stats["elements_valid"], 1),

@@ -85,8 +85,10 @@ int hpctopk_version(void);
 const char* hpctopk_status_string(int status);
 
 /* Bytes of device workspace hpctopk_select needs for up to `max_num_rows` rows at rank K.
- * Bounded by a constant plus 16 bytes per row (independent of row width; Section 2.1,
- * "Deployment requirements").  Host only.  Returns 0 for invalid arguments. */
+ * Independent of row width (Section 2.1, "Deployment requirements"): a constant plus 16 bytes
+ * per row, plus - for calls of 513 to 8192 rows, which run as three kernels - one candidate
+ * range of max(4K, 4096) 8-byte entries per row (64 KB per row at K = 2048).  Host only.
+ * Returns 0 for invalid arguments. */
 size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K);
 
 /* Policy the selector applies at rank K to a row of valid length L (host mirror of the
@@ -97,6 +99,11 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K);
  *               "enters the sampled path"
  * Any output pointer may be NULL.  Host only. */
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route);
+
+/* Number of kernels one hpctopk_select call of `num_rows` rows launches on the current device
+ * (1: the single persistent kernel; 3: boundary, pass and refinement kernels).  Host only;
+ * returns 0 for num_rows <= 0. */
+int hpctopk_kernels_per_call(int32_t num_rows);
 
 /* Exact Top-K of every row (operator contract, Section 2.1; phases of Sections 4.2-4.4).
  *
@@ -116,9 +123,9 @@ int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacit
  *   workspace   >= hpctopk_workspace_bytes(num_rows, K) bytes, 256-byte aligned; contents
  *               need not be initialised; calls that may overlap on the device need
  *               distinct workspaces
- *   stream      all work is enqueued on `stream` (one small memset and one kernel whose
- *               launch geometry depends only on num_rows, K and the device); nothing is
- *               read back, so the call can be captured in a CUDA graph and replayed with
+ *   stream      all work is enqueued on `stream` (one small memset and one or three kernels
+ *               whose launch geometry depends only on num_rows, K and the device); nothing
+ *               is read back, so the call can be captured in a CUDA graph and replayed with
  *               new contents in the same buffers.  The very first call on a device also
  *               fills a 8 KB lookup table and synchronises the device once: make it
  *               outside any capture
@@ -127,6 +134,17 @@ int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacit
 int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
                    int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
                    void* workspace, hpctopk_stream_t stream);
+
+/* Measurement aid (no counterpart in the paper): device time of the dominant kernel of each
+ * call - the pass kernel of a three-kernel call, the one kernel otherwise - taken with CUDA
+ * events recorded on the call's stream right before and after that launch.
+ *   hpctopk_stage_timing(1) creates the events for the current device (first use) and switches
+ *   the recording on, hpctopk_stage_timing(0) switches it off.  Calls made while the stream is
+ *   being captured are not timed.  At most 1024 calls are kept between two reads.
+ *   hpctopk_read_stage_timing waits for the recorded events, returns the summed milliseconds
+ *   and the number of calls they cover, and starts a new interval.  Host only; not thread-safe. */
+int hpctopk_stage_timing(int enable);
+int hpctopk_read_stage_timing(float* total_ms, int32_t* calls);
 
 /* Enqueue a copy of the workspace's counters into `host_out` (host memory).  The caller
  * synchronises `stream` before reading.  Section 4.5 defines the rates these counters

@@ -59,6 +59,10 @@ def lib():
         L.hpctopk_workspace_bytes.argtypes = [i32, i32]
         L.hpctopk_workspace_bytes.restype = ctypes.c_size_t
         L.hpctopk_query_policy.argtypes = [i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.hpctopk_stage_timing.argtypes = [ctypes.c_int]
+        L.hpctopk_read_stage_timing.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
+        L.hpctopk_kernels_per_call.argtypes = [i32]
+        L.hpctopk_kernels_per_call.restype = ctypes.c_int
         L.hpctopk_query_policy.restype = ctypes.c_int
         L.hpctopk_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.hpctopk_select.restype = ctypes.c_int
@@ -97,6 +101,27 @@ def hpctopk_query_policy(K, L):
     if st != HPCTOPK_OK:
         raise HpcTopkError(st)
     return s.value, c.value, r.value
+
+
+def hpctopk_kernels_per_call(num_rows):
+    """Kernels one hpctopk_select call of ``num_rows`` rows launches (1 or 3)."""
+    return int(lib().hpctopk_kernels_per_call(int(num_rows)))
+
+
+def hpctopk_stage_timing(enable):
+    """Switch the event timing of each call's dominant kernel on or off (current device)."""
+    st = lib().hpctopk_stage_timing(1 if enable else 0)
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+
+
+def hpctopk_read_stage_timing():
+    """(total milliseconds, calls) of the dominant kernel since the last read."""
+    ms, n = ctypes.c_float(), ctypes.c_int32()
+    st = lib().hpctopk_read_stage_timing(ctypes.byref(ms), ctypes.byref(n))
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    return ms.value, n.value
 
 
 def hpctopk_select_raw(scores_ptr, row_starts_ptr, row_lengths_ptr, num_rows, K, out_idx_ptr,

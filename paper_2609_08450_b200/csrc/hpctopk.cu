@@ -1450,6 +1450,7 @@ constexpr int kDefaultVariant = kPipeVariant;
 constexpr int kMonoVariant = 4;
 constexpr int kSplitVariant = 1;
 constexpr int kPipeRowsMax = 8192;
+constexpr int kTimingSlots = 1024;
 constexpr int kBoundaryThreads = 128;
 #ifndef HPCTOPK_REFINE_T
 #define HPCTOPK_REFINE_T 128
@@ -1464,6 +1465,9 @@ struct DeviceInfo {
   int variant = 0;      // 0: warp-specialised kernel; v >= 1: single-role kernel kVariants[v - 1]
   int ctas_per_sm[2][3] = {{0, 0, 0}, {0, 0, 0}};   // [split][capacity class]
   int boundary_per_sm = 0;                          // pipeline: boundary kernel
+  bool timing = false;                              // hpctopk_stage_timing
+  int timed = 0;                                    // event pairs recorded since the last read
+  cudaEvent_t ev0[kTimingSlots] = {}, ev1[kTimingSlots] = {};
   int pipe_stages = 3;                              // tuning: run only the first n kernels (HPCTOPK_PIPE_STAGES)
 };
 DeviceInfo g_dev[64];
@@ -1501,14 +1505,61 @@ PipeLayout pipe_layout(int rows, int K) {
   return l;
 }
 
-const auto kPassKernel = pipe_pass_kernel<512, 2, 3>;
-constexpr int kPassThreads = 512;
+#ifndef HPCTOPK_PASS_T
+#define HPCTOPK_PASS_T 512
+#define HPCTOPK_PASS_MINB 3
+#endif
+const auto kPassKernel = pipe_pass_kernel<HPCTOPK_PASS_T, 2, HPCTOPK_PASS_MINB>;
+constexpr int kPassThreads = HPCTOPK_PASS_T;
 const auto kRefineKernel = pipe_refine_kernel<kRefineThreads, 2, HPCTOPK_REFINE_MINB>;
 const auto kBoundaryKernel = pipe_boundary_kernel<kBoundaryThreads>;
+
+// Event pair for this call, or -1 when stage timing is off, full, or the stream is being captured.
+int timing_slot(DeviceInfo& di, cudaStream_t st) {
+  if (!di.timing || di.timed >= kTimingSlots) return -1;
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) { cudaGetLastError(); return -1; }
+  return di.timed++;
+}
 
 }  // namespace
 
 extern "C" {
+
+int hpctopk_stage_timing(int enable) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HPCTOPK_ERR_CUDA;
+  DeviceInfo& di = g_dev[dev];
+  if (enable && !di.ev0[0]) {
+    for (int i = 0; i < kTimingSlots; ++i)
+      if (cudaEventCreate(&di.ev0[i]) != cudaSuccess || cudaEventCreate(&di.ev1[i]) != cudaSuccess) {
+        cudaGetLastError();
+        return HPCTOPK_ERR_CUDA;
+      }
+  }
+  di.timing = enable != 0;
+  return HPCTOPK_OK;
+}
+
+int hpctopk_read_stage_timing(float* total_ms, int32_t* calls) {
+  if (!total_ms || !calls) return HPCTOPK_ERR_INVALID_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HPCTOPK_ERR_CUDA;
+  DeviceInfo& di = g_dev[dev];
+  float sum = 0.f;
+  for (int i = 0; i < di.timed; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(di.ev1[i]) != cudaSuccess || cudaEventElapsedTime(&ms, di.ev0[i], di.ev1[i]) != cudaSuccess) {
+      cudaGetLastError();
+      return HPCTOPK_ERR_CUDA;
+    }
+    sum += ms;
+  }
+  *total_ms = sum;
+  *calls = di.timed;
+  di.timed = 0;
+  return HPCTOPK_OK;
+}
 
 int hpctopk_version(void) { return 1000 * 0 + 1; }
 
@@ -1545,6 +1596,13 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
     if (p > b) b = p;
   }
   return b;
+}
+
+int hpctopk_kernels_per_call(int32_t num_rows) {
+  if (num_rows <= 0) return 0;
+  const char* env = getenv("HPCTOPK_VARIANT");
+  const int variant = env ? atoi(env) : kDefaultVariant;
+  return (variant == kPipeVariant && num_rows > kSplitRowsMax && num_rows <= kPipeRowsMax) ? 3 : 1;
 }
 
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route) {
@@ -1649,7 +1707,10 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     int g1 = di.sm_count * di.boundary_per_sm;
     if (g1 > num_rows) g1 = num_rows;
     kBoundaryKernel<<<g1, kBoundaryThreads, smem_small, st>>>(P);
+    const int slot = timing_slot(di, st);
+    if (slot >= 0) cudaEventRecord(di.ev0[slot], st);
     if (di.pipe_stages >= 2) kPassKernel<<<num_rows, kPassThreads, smem_pass, st>>>(P);
+    if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
     Params R = P;
     R.cap_s = 0;
     if (di.pipe_stages >= 3) kRefineKernel<<<num_rows, kRefineThreads, smem_small, st>>>(R);
@@ -1667,7 +1728,10 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     int ws_grid = di.sm_count < wsk::kWsMaxGrid ? di.sm_count : wsk::kWsMaxGrid;
     wsk::hpctopk_ws_kernel<wsk::kWsU><<<ws_grid, wsk::THREADS, wsk::ws_smem_bytes(K, split), st>>>(P);
   } else {
+    const int slot = timing_slot(di, st);
+    if (slot >= 0) cudaEventRecord(di.ev0[slot], st);
     v.fn<<<grid, v.threads, smem, st>>>(P);
+    if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
   }
   if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
   return HPCTOPK_OK;

@@ -22,7 +22,8 @@ def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "hpctopk.h")).read()
     names = set(re.findall(r"\b(hpctopk_[a-z_]+)\s*\(", header))
     assert {"hpctopk_select", "hpctopk_workspace_bytes", "hpctopk_read_stats", "hpctopk_read_row_info",
-            "hpctopk_query_policy", "hpctopk_status_string", "hpctopk_version"} <= names
+            "hpctopk_query_policy", "hpctopk_kernels_per_call", "hpctopk_status_string",
+            "hpctopk_version"} <= names
     for n in names:
         assert hasattr(lib, n), n
 
@@ -51,6 +52,8 @@ def test_policy_mirror_matches_the_reading_of_the_paper(lib):
     assert B.hpctopk_query_policy(2048, 1)[0] == 128
     with pytest.raises(B.HpcTopkError):
         B.hpctopk_query_policy(0, 5)
+    if "HPCTOPK_VARIANT" not in os.environ:
+        assert [B.hpctopk_kernels_per_call(m) for m in (0, 1, 512, 513, 8192, 8193)] == [0, 1, 1, 3, 3, 1]
 
 
 def test_argument_validation_returns_before_any_cuda_call(lib):

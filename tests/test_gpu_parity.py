@@ -140,17 +140,18 @@ def test_negative_and_zero_lengths_are_empty_rows():
     _common().check_batch(batch, 16)
 
 
-def test_cuda_graph_replay_with_new_lengths_in_the_same_buffers():
+@pytest.mark.parametrize("M,max_len", [(24, 90000), (600, 30000)])     # single kernel; three-kernel pipeline
+def test_cuda_graph_replay_with_new_lengths_in_the_same_buffers(M, max_len):
     K = 2048
-    a = W.config1(DEV, seed=11, num_rows=24, max_len=90000)
-    b = W.config1(DEV, seed=12, num_rows=24, max_len=90000)
+    a = W.config1(DEV, seed=11, num_rows=M, max_len=max_len)
+    b = W.config1(DEV, seed=12, num_rows=M, max_len=max_len)
     n = max(a.scores.numel(), b.scores.numel())
     scores = torch.zeros(n, device=DEV)
-    starts = torch.zeros(24, dtype=torch.int32, device=DEV)
-    lengths = torch.zeros(24, dtype=torch.int32, device=DEV)
-    out_idx = torch.empty((24, K), dtype=torch.int32, device=DEV)
-    out_val = torch.empty((24, K), dtype=torch.float32, device=DEV)
-    ws = torch.empty(B.hpctopk_workspace_bytes(24, K), dtype=torch.uint8, device=DEV)
+    starts = torch.zeros(M, dtype=torch.int32, device=DEV)
+    lengths = torch.zeros(M, dtype=torch.int32, device=DEV)
+    out_idx = torch.empty((M, K), dtype=torch.int32, device=DEV)
+    out_val = torch.empty((M, K), dtype=torch.float32, device=DEV)
+    ws = torch.empty(B.hpctopk_workspace_bytes(M, K), dtype=torch.uint8, device=DEV)
 
     def load(batch):
         scores[: batch.scores.numel()].copy_(batch.scores)
