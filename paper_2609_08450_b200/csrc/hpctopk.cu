@@ -792,9 +792,15 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
 // ranking its members against each other under (kd, idx).  Returns false, with nothing written,
 // when the K-th score falls outside the bracket or the boundary bin is too large: the caller
 // then runs the general 11+11+10 refinement.
-template <int THREADS, bool BLOCK_SEARCH = false, bool COUNT0 = false>
+// STAGE_OUT: the K results are collected in the shared memory behind the kernel's Shared block
+// (2 x K words, which the launch must provide) and written out as whole lines at the end; the
+// commit pass otherwise scatters 4-byte stores over the output row, which cost the refinement
+// kernel a third of its time.
+template <int THREADS, bool BLOCK_SEARCH = false, bool COUNT0 = false, bool STAGE_OUT = false>
 __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint32_t K, uint32_t cut_base, uint32_t cut_hi,
                                              int32_t* out_idx, float* out_val, uint32_t cut_count = 0u) {
+  int32_t* const w_idx = STAGE_OUT ? reinterpret_cast<int32_t*>(CAND()) : out_idx;
+  float* const w_val = STAGE_OUT ? reinterpret_cast<float*>(CAND()) + K : out_val;
   Shared& sh = SH();
   constexpr int W = THREADS <= 128 ? 8 : 4;      // entries per thread and batch (independent loads in flight)
   const int tid = threadIdx.x, lane = tid & 31;
@@ -871,7 +877,7 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
 #pragma unroll
     for (int k = 0; k < W; ++k) {
       if (dg[k] < (uint32_t)b) {
-        if (pos < K) { out_idx[pos] = (int32_t)c[k].y; if (out_val) out_val[pos] = __uint_as_float(bits_of_kd(c[k].x)); }
+        if (pos < K) { w_idx[pos] = (int32_t)c[k].y; if (w_val) w_val[pos] = __uint_as_float(bits_of_kd(c[k].x)); }
         ++pos;
       } else if (dg[k] == (uint32_t)b) {
         const uint32_t lp = atomicAdd(&sh.small_count, 1u);
@@ -890,11 +896,15 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
       rank += ((((uint64_t)o.x << 32) | o.y) < mine) ? 1u : 0u;
     }
     if (rank < k_rem) {
-      out_idx[below + rank] = (int32_t)me.y;
-      if (out_val) out_val[below + rank] = __uint_as_float(bits_of_kd(me.x));
+      w_idx[below + rank] = (int32_t)me.y;
+      if (w_val) w_val[below + rank] = __uint_as_float(bits_of_kd(me.x));
     }
   }
   __syncthreads();
+  if (STAGE_OUT) {
+    for (uint32_t i = tid; i < K; i += THREADS) out_idx[i] = w_idx[i];
+    if (out_val) for (uint32_t i = tid; i < K; i += THREADS) out_val[i] = w_val[i];
+  }
   DSTAMP(4, ts);
   return true;
 }
@@ -1377,7 +1387,7 @@ __global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params
         // entries, so the whole stored tail is refined against its own cutoff and C(tau_0) is
         // only counted (for the route the row reports).
         const uint32_t cut_base = band2 ? sh.cutd[3] : sh.cutd[1];
-        if (!select_adaptive<THREADS, true, true>(rc, C1, K, cut_base, sh.cutd[2], oi, ov, sh.cutd[0])) {
+        if (!select_adaptive<THREADS, true, true, true>(rc, C1, K, cut_base, sh.cutd[2], oi, ov, sh.cutd[0])) {
           if (tid == 0) add64(&stats_of(P.ws)->general_refinements, 1);
           __syncthreads();
           CandidateSource cs{rc, C1, cut_base};
@@ -1713,7 +1723,7 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
     Params R = P;
     R.cap_s = 0;
-    if (di.pipe_stages >= 3) kRefineKernel<<<num_rows, kRefineThreads, smem_small, st>>>(R);
+    if (di.pipe_stages >= 3) kRefineKernel<<<num_rows, kRefineThreads, smem_bytes_for(K, false), st>>>(R);   // + 2K words of output staging
   } else if (di.variant == kFusedVariant) {
     const size_t fsmem = wsf::ws_smem_bytes(K, split);
     int per_sm = 0;
