@@ -101,7 +101,8 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K);
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route);
 
 /* Number of kernels one hpctopk_select call of `num_rows` rows launches on the current device
- * (1: the single persistent kernel; 3: boundary, pass and refinement kernels).  Host only;
+ * (1: the single persistent kernel; 3: boundary, pass and refinement kernels, calls of 513 to
+ * 8192 rows).  Host only;
  * returns 0 for num_rows <= 0. */
 int hpctopk_kernels_per_call(int32_t num_rows);
 

@@ -784,6 +784,22 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   return true;
 }
 
+// The row's boundary: read from the record a boundary kernel left (when the call ran one), else
+// computed here.  Leaves the cutoffs in sh.cutd like phase1; contains block barriers.
+__device__ __forceinline__ RowRec* pipe_rec(const Params& P) { return reinterpret_cast<RowRec*>(P.ws + P.pipe_rec_off); }
+template <int THREADS>
+__device__ __forceinline__ bool row_boundary(const Params& P, int row, int64_t g0, int64_t L, int& tau_pack) {
+  if (P.pipe_rec_off == 0) return phase1<THREADS>(P, row, g0, L, tau_pack);
+  Shared& sh = SH();
+  const RowRec* rec = pipe_rec(P) + row;
+  __syncthreads();
+  if (threadIdx.x < 4) sh.cutd[threadIdx.x] = __ldg(&rec->cutd[threadIdx.x]);
+  tau_pack = __ldg(&rec->tau_pack);
+  const bool usable = __ldg(&rec->usable) != 0u;
+  __syncthreads();
+  return usable;
+}
+
 // Phase 3 with a row-adaptive first digit (any monotone digit of the key is a valid refinement
 // digit, Section 4.4): d = min((cut_base - kd) >> sh, 2047) measures the distance from the
 // admitted cutoff in units of 2^sh ulps, with sh chosen so that the bracket [cut_hi, cut_base]
@@ -1010,7 +1026,7 @@ __device__ void process_row(const Params& P, int row, const CandCtx cc) {
   }
   int tau_pack;
   const long long t0 = tick();
-  if (!phase1<THREADS>(P, row, g0, L, tau_pack)) {
+  if (!row_boundary<THREADS>(P, row, g0, L, tau_pack)) {
     RowSource rs{P.scores, g0, g0 + L};
     select_and_emit<THREADS>(rs, K, false, oi, ov);
     record_row(P, row, HPCTOPK_ROUTE_RECOVERY, -1, 0, 0, 4ull * (uint64_t)L, 0, (uint64_t)L);
@@ -1050,9 +1066,10 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
 
   int tau_pack;
   const long long t0 = tick();
-  const bool usable = phase1<THREADS>(P, row, g0, L, tau_pack);
+  const bool usable = row_boundary<THREADS>(P, row, g0, L, tau_pack);
   const long long t1 = tick();
-  const uint64_t sampled = usable ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
+  // the view is read once per row when a boundary kernel ran, once per segment otherwise
+  const uint64_t sampled = usable && (P.pipe_rec_off == 0 || seg == 0) ? (uint64_t)((L + P.stride - 1) / P.stride) : 0;
   // contiguous, 16-byte aligned partition of the row's vectors
   const int64_t va = g0 >> 2, vb = (g1 + 3) >> 2;
   const int64_t per = (vb - va + nseg - 1) / nseg;
@@ -1258,7 +1275,6 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
 // time and the short phases run at their own, higher occupancy.  Cost: the admitted tails cross
 // HBM once each way (about 57 KB per row at K = 2048, 11 % of a 129 K-score row).
 constexpr uint32_t kBand2Flag = 0x80000000u;    // in a row's admitted count: the tail includes the second band
-__device__ __forceinline__ RowRec* pipe_rec(const Params& P) { return reinterpret_cast<RowRec*>(P.ws + P.pipe_rec_off); }
 __device__ __forceinline__ uint32_t* pipe_cnt(const Params& P) { return reinterpret_cast<uint32_t*>(P.ws + P.pipe_cnt_off); }
 __device__ __forceinline__ uint2* pipe_cand(const Params& P, int row) {
   return reinterpret_cast<uint2*>(P.ws + P.pipe_cand_off) + (size_t)row * (size_t)P.cap;
@@ -1738,6 +1754,9 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
     int ws_grid = di.sm_count < wsk::kWsMaxGrid ? di.sm_count : wsk::kWsMaxGrid;
     wsk::hpctopk_ws_kernel<wsk::kWsU><<<ws_grid, wsk::THREADS, wsk::ws_smem_bytes(K, split), st>>>(P);
   } else {
+    // (A boundary kernel in front of a split call, so that Phase 1 runs once per row instead of
+    // once per segment, was measured: the segments' Phase 1 run side by side anyway and the extra
+    // launch is serial - config 2 went from 58 to 71 us, config 4 from 75 to 69 us.  Left out.)
     const int slot = timing_slot(di, st);
     if (slot >= 0) cudaEventRecord(di.ev0[slot], st);
     v.fn<<<grid, v.threads, smem, st>>>(P);

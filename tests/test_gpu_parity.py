@@ -176,3 +176,21 @@ def test_cuda_graph_replay_with_new_lengths_in_the_same_buffers(M, max_len):
         s, st, ln = batch.host()
         want, _, _ = native.topk_stable_sort(s, st, ln, K)
         assert_rows_match(s, st, ln, K, out_idx.cpu().numpy(), out_val.cpu().numpy(), want)
+
+
+def test_stage_timing_reports_the_dominant_kernel():
+    """The measurement aid of the C ABI: one event pair per call around the kernel that reads
+    every score; the call's results are unaffected."""
+    K = 1024
+    batch = W.config1(DEV, seed=21, num_rows=600, max_len=20000, K=K)     # three-kernel call
+    assert B.hpctopk_kernels_per_call(batch.num_rows) == 3
+    B.hpctopk_stage_timing(True)
+    B.hpctopk_read_stage_timing()
+    try:
+        for _ in range(3):
+            _common().check_batch(batch, K)
+        ms, calls = B.hpctopk_read_stage_timing()
+    finally:
+        B.hpctopk_stage_timing(False)
+    assert calls == 3 and 0.0 < ms < 1000.0
+    assert B.hpctopk_read_stage_timing() == (0.0, 0)
