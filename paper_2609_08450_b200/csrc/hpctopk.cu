@@ -44,7 +44,7 @@ __device__ __forceinline__ long long tick() {
 constexpr int kBins = 2048;            // B_c and the widest refinement digit
 constexpr int kSplitRowsMax = 512;     // rows beyond this are never split (enough row parallelism)
 constexpr int kSegMinElems = 16384;    // shortest segment worth a CTA
-constexpr int kTasksPerCta = 2;        // split target: tasks >= kTasksPerCta * grid
+constexpr int kTasksPerCta = 1;        // split target: tasks >= kTasksPerCta * grid
 constexpr int kSmallMax = kBins / 2;   // boundary group resolved by direct ranking (pairs held in the histogram's memory)
 
 // workspace layout (bytes)
@@ -1164,8 +1164,9 @@ __device__ __forceinline__ int row_of_task(const Params& P, uint32_t task) {
 
 // Device-side ragged dispatch (Section 4.5): every CTA derives the same task table from
 // row_lengths.  seg_base[r] is the first task of row r, seg_base[num_rows] the task count; a long
-// row gets ceil(L / S) segment tasks with S = max(16384, total / (grid * kTasksPerCta)) rounded
-// up to 4096 elements, every other row one task.  Contains block barriers.
+// row gets ceil(L / S) segment tasks with S = max(16384, total / (grid' * kTasksPerCta)) rounded
+// up to 4096 elements (grid' = grid minus the number of long rows), every other row one task.
+// Contains block barriers.
 template <int THREADS>
 __device__ uint32_t build_task_table(const Params& P, uint32_t* seg_base) {
   Shared& sh = SH();
@@ -1174,14 +1175,19 @@ __device__ uint32_t build_task_table(const Params& P, uint32_t* seg_base) {
   unsigned long long mine = 0;
   for (int j = 0; j < RPT; ++j) {
     const int r = tid * RPT + j;
-    if (r < P.num_rows) { const int64_t L = P.row_lengths[r]; if (L > P.cap) mine += (unsigned long long)L; }
+    if (r < P.num_rows) { const int64_t L = P.row_lengths[r]; if (L > P.cap) mine += (unsigned long long)L + (1ull << 50); }   // length sum, row count above bit 50
   }
   for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
   if ((tid & 31) == 0) { sh.hist[2 * (tid >> 5)] = (uint32_t)mine; sh.hist[2 * (tid >> 5) + 1] = (uint32_t)(mine >> 32); }
   __syncthreads();
   unsigned long long total = 0;
   for (int w = 0; w < THREADS / 32; ++w) total += (unsigned long long)sh.hist[2 * w] | ((unsigned long long)sh.hist[2 * w + 1] << 32);
-  const unsigned long long target = (unsigned long long)gridDim.x * kTasksPerCta;
+  // one task per CTA, so that a row's boundary (recomputed by every segment's CTA) is on the
+  // critical path once; every long row may add one partial segment, hence the correction
+  const unsigned long long nlong = total >> 50;
+  total &= (1ull << 50) - 1ull;
+  unsigned long long target = (unsigned long long)gridDim.x * kTasksPerCta;
+  if (target > 2ull * nlong) target -= nlong;
   unsigned long long S = (total + target - 1) / target;
   if (S < (unsigned long long)kSegMinElems) S = kSegMinElems;
   S = (S + 4095ull) / 4096ull * 4096ull;
