@@ -310,6 +310,17 @@ def main():
             line["cpu_baseline"] = {"value": ne / dt, "unit": "score elements/s", "cores": used, "kind": "oracle",
                                     "sample": f"{len(rows)} evenly spaced rows of the workload ({ne} score elements), "
                                               f"std::stable_sort per row, OpenMP over rows"}
+            # beside it: one thread, and the oracle's O(L) std::nth_element selector on all threads
+            # (a 64-row sample each, a few seconds)
+            from oracle import native
+            few = oracle_sample_rows(M, min(64, len(rows)))
+            n_few = int(np.clip(lengths[few], 0, None).sum())
+            t0 = time.perf_counter()
+            native.topk_stable_sort(scores, starts[few], lengths[few], K, num_threads=1)
+            line["cpu_baseline"]["single_thread_value"] = n_few / (time.perf_counter() - t0)
+            t0 = time.perf_counter()
+            native.topk_nth_element(scores, starts[few], lengths[few], K)
+            line["cpu_baseline"]["nth_element_value"] = n_few / (time.perf_counter() - t0)
         else:
             line["cpu_baseline"] = None
         print(json.dumps(line), flush=True)

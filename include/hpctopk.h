@@ -136,6 +136,16 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
                    int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
                    void* workspace, hpctopk_stream_t stream);
 
+/* The same operator on the padded matrix of the paper's contract (Section 2.1: M rows of a
+ * common pitch with per-row valid lengths): row r starts at `scores + r * pitch` (pitch in
+ * elements, >= every valid length; r * pitch may exceed 2^31).  A pitch that is a multiple of 4
+ * keeps every row 16-byte aligned, which removes the scalar edge handling of packed rows.
+ * All other arguments, the output layout, the workspace size and the error behaviour are those
+ * of hpctopk_select; pitch < 0 returns HPCTOPK_ERR_INVALID_ARG. */
+int hpctopk_select_padded(const float* scores, int64_t pitch, const int32_t* row_lengths,
+                          int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                          void* workspace, hpctopk_stream_t stream);
+
 /* Measurement aid (no counterpart in the paper): device time of the dominant kernel of each
  * call - the pass kernel of a three-kernel call, the one kernel otherwise - taken with CUDA
  * events recorded on the call's stream right before and after that launch.

@@ -66,6 +66,8 @@ def lib():
         L.hpctopk_query_policy.restype = ctypes.c_int
         L.hpctopk_select.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp]
         L.hpctopk_select.restype = ctypes.c_int
+        L.hpctopk_select_padded.argtypes = [vp, i64, vp, i32, i32, vp, vp, vp, vp]
+        L.hpctopk_select_padded.restype = ctypes.c_int
         L.hpctopk_select_static.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
         L.hpctopk_select_static.restype = ctypes.c_int
         L.hpctopk_read_stats.argtypes = [vp, ctypes.POINTER(Stats), vp]
@@ -155,6 +157,38 @@ def hpctopk_select(scores, row_starts, row_lengths, K, out_idx=None, out_val=Non
         st = hpctopk_select_raw(scores.data_ptr(), row_starts.data_ptr(), row_lengths.data_ptr(), M, K,
                                 out_idx.data_ptr(), out_val.data_ptr() if out_val is not None else None,
                                 workspace.data_ptr(), stream.cuda_stream)
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
+    return out_idx, out_val, workspace
+
+
+def hpctopk_select_padded(matrix, row_lengths, K, out_idx=None, out_val=None, workspace=None, stream=None,
+                          want_values=True):
+    """Select on a padded [M, pitch] fp32 CUDA matrix (row r valid up to row_lengths[r]).
+
+    ``matrix`` may be a row-strided view: its row stride is the pitch, its column stride must be 1.
+    Returns (out_idx [M, K] int32, out_val [M, K] fp32 or None, workspace uint8 tensor).
+    """
+    import torch
+    assert matrix.is_cuda and matrix.dtype == torch.float32 and matrix.dim() == 2
+    assert matrix.size(1) <= 1 or matrix.stride(1) == 1
+    assert row_lengths.dtype == torch.int32
+    M = int(matrix.size(0))
+    assert int(row_lengths.numel()) == M
+    pitch = int(matrix.stride(0)) if M > 1 else int(matrix.size(1))
+    dev = matrix.device
+    if out_idx is None:
+        out_idx = torch.empty((M, K), dtype=torch.int32, device=dev)
+    if out_val is None and want_values:
+        out_val = torch.empty((M, K), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(max(hpctopk_workspace_bytes(M, K), 256), dtype=torch.uint8, device=dev)
+    if stream is None:
+        stream = torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        st = int(lib().hpctopk_select_padded(matrix.data_ptr(), pitch, row_lengths.data_ptr(), M, int(K),
+                                             out_idx.data_ptr(), out_val.data_ptr() if out_val is not None else None,
+                                             workspace.data_ptr(), stream.cuda_stream))
     if st != HPCTOPK_OK:
         raise HpcTopkError(st)
     return out_idx, out_val, workspace

@@ -76,7 +76,8 @@ __host__ __device__ inline int stride_for(int K) {
 
 struct Params {
   const float* scores;
-  const int32_t* row_starts;
+  const int32_t* row_starts;    // NULL: padded matrix, row r starts at element r * pitch
+  int64_t pitch;
   const int32_t* row_lengths;
   int32_t num_rows;
   int32_t K;
@@ -102,6 +103,11 @@ struct RowRec {
   uint32_t pad[2];
 };
 static_assert(sizeof(RowRec) == 32, "RowRec is read as two 16-byte vectors");
+
+// Element offset of row r in `scores`.
+__device__ __forceinline__ int64_t row_start(const Params& P, int row) {
+  return P.row_starts ? (int64_t)P.row_starts[row] : (int64_t)row * P.pitch;
+}
 
 struct Shared {
   hpctopk_stats acc;         // this CTA's counters (first member of every kernel's shared state)
@@ -1000,7 +1006,7 @@ __device__ void finish_sampled_row(const Params& P, const CandCtx cc, int row, i
 template <int THREADS, int U>
 __device__ void process_row(const Params& P, int row, const CandCtx cc) {
   Shared& sh = SH();
-  const int64_t g0 = P.row_starts[row];
+  const int64_t g0 = row_start(P, row);
   int64_t L = P.row_lengths[row];
   if (L < 0) L = 0;
   const uint32_t K = (uint32_t)P.K, cap = (uint32_t)P.cap;
@@ -1055,7 +1061,7 @@ template <int THREADS, int U>
 __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
   Shared& sh = SH();
   const CandCtx cc = cand_ctx(P);
-  const int64_t g0 = P.row_starts[row];
+  const int64_t g0 = row_start(P, row);
   const int64_t L = P.row_lengths[row];       // > cap, checked when the table was built
   const int64_t g1 = g0 + L;
   const uint32_t cap = (uint32_t)P.cap;
@@ -1134,7 +1140,7 @@ __device__ void process_segment(const Params& P, int row, int seg, int nseg) {
 // not start with a DRAM round trip.
 template <int THREADS>
 __device__ __forceinline__ void prefetch_view(const Params& P, int row) {
-  const int64_t g0 = P.row_starts[row];
+  const int64_t g0 = row_start(P, row);
   const int64_t L = P.row_lengths[row];
   if (L <= P.cap) return;
   const int s = P.stride;
@@ -1242,7 +1248,7 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
     if (!P.split_enabled && next < total_tasks) {
       const int nrow = row_of_task(P, next);
       prefetch_view<THREADS>(P, nrow);
-      const int64_t ng0 = P.row_starts[nrow], nL = P.row_lengths[nrow];
+      const int64_t ng0 = row_start(P, nrow), nL = P.row_lengths[nrow];
       if (nL > P.K) prefetch_head<THREADS>(P, ng0, ng0 + nL);
     }
     if (P.split_enabled) {
@@ -1292,7 +1298,7 @@ __global__ void __launch_bounds__(THREADS) pipe_boundary_kernel(const Params P) 
   stats_clear();
   __syncthreads();
   for (int row = P.row_begin + blockIdx.x; row < P.row_end; row += gridDim.x) {
-    const int64_t g0 = P.row_starts[row];
+    const int64_t g0 = row_start(P, row);
     const int64_t L = P.row_lengths[row];
     int tau_pack = -1;
     bool usable = false;
@@ -1316,7 +1322,7 @@ __device__ void pipe_pass_task(const Params& P, int row) {
   // entries beyond the on-chip part go straight to their place in the row's global range
   CandCtx cc;
   cc.cap_s = (uint32_t)P.cap_s; cc.cap = (uint32_t)P.cap; cc.spill = pipe_cand(P, row) + P.cap_s;
-  const int64_t g0 = P.row_starts[row];
+  const int64_t g0 = row_start(P, row);
   const int64_t L = P.row_lengths[row];
   if (L <= (int64_t)P.cap) return;                       // short and direct rows: refinement kernel
   const RowRec* rec = pipe_rec(P) + row;
@@ -1382,7 +1388,7 @@ __global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params
   __syncthreads();
   {
     const int row = P.row_end - 1 - (int)blockIdx.x;
-    const int64_t g0 = P.row_starts[row];
+    const int64_t g0 = row_start(P, row);
     const int64_t L = P.row_lengths[row];
     const RowRec* rec = pipe_rec(P) + row;
     const bool sampled = L > (int64_t)cap && __ldg(&rec->usable) != 0u;
@@ -1646,13 +1652,31 @@ int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacit
   return HPCTOPK_OK;
 }
 
+static int select_impl(const float* scores, const int32_t* row_starts, int64_t pitch, const int32_t* row_lengths,
+                       int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                       void* workspace, hpctopk_stream_t stream);
+
 int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t* row_lengths,
                    int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
                    void* workspace, hpctopk_stream_t stream) {
+  if (num_rows > 0 && !row_starts) return HPCTOPK_ERR_INVALID_ARG;
+  return select_impl(scores, row_starts, 0, row_lengths, num_rows, K, out_idx, out_val, workspace, stream);
+}
+
+int hpctopk_select_padded(const float* scores, int64_t pitch, const int32_t* row_lengths,
+                          int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                          void* workspace, hpctopk_stream_t stream) {
+  if (pitch < 0) return HPCTOPK_ERR_INVALID_ARG;
+  return select_impl(scores, nullptr, pitch, row_lengths, num_rows, K, out_idx, out_val, workspace, stream);
+}
+
+static int select_impl(const float* scores, const int32_t* row_starts, int64_t pitch, const int32_t* row_lengths,
+                       int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
+                       void* workspace, hpctopk_stream_t stream) {
   if (num_rows < 0 || K < 1) return HPCTOPK_ERR_INVALID_ARG;
   if (K > HPCTOPK_MAX_K) return HPCTOPK_ERR_UNSUPPORTED_K;
   if (num_rows == 0) return HPCTOPK_OK;
-  if (!scores || !row_starts || !row_lengths || !out_idx || !workspace) return HPCTOPK_ERR_INVALID_ARG;
+  if (!scores || !row_lengths || !out_idx || !workspace) return HPCTOPK_ERR_INVALID_ARG;
   if (((uintptr_t)scores & 15u) || ((uintptr_t)workspace & 255u)) return HPCTOPK_ERR_MISALIGNED;
 
   int dev = 0;
@@ -1708,7 +1732,7 @@ int hpctopk_select(const float* scores, const int32_t* row_starts, const int32_t
   const Variant& v = kVariants[variant_index(di.variant, split)];
   const int cls = cap_class(K);
   Params P;
-  P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
+  P.scores = scores; P.row_starts = row_starts; P.pitch = pitch; P.row_lengths = row_lengths;
   P.num_rows = num_rows; P.K = K; P.out_idx = out_idx; P.out_val = out_val;
   P.ws = static_cast<unsigned char*>(workspace);
   P.cap = capacity_for(K);
@@ -1852,7 +1876,7 @@ extern "C" int hpctopk_select_static(const float* scores, const int32_t* row_sta
   }
   const int cls = cap_class(K);
   Params P;
-  P.scores = scores; P.row_starts = row_starts; P.row_lengths = row_lengths;
+  P.scores = scores; P.row_starts = row_starts; P.pitch = 0; P.row_lengths = row_lengths;
   P.num_rows = num_rows; P.K = K; P.out_idx = out_idx; P.out_val = out_val;
   P.ws = static_cast<unsigned char*>(g_static_scratch_addr[dev]);
   P.cap = capacity_for(K);

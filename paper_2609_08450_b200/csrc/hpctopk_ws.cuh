@@ -950,7 +950,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
         nseg = (int)(seg_base[row + 1] - seg_base[row]);
         seg = (int)(task - seg_base[row]);
       }
-      const int64_t g0 = P.row_starts[row];
+      const int64_t g0 = row_start(P, row);
       int64_t L = P.row_lengths[row];
       if (L < 0) L = 0;
       t.row = row; t.seg = seg; t.nseg = nseg; t.g0 = g0; t.L = L;

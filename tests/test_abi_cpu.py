@@ -22,7 +22,7 @@ def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "hpctopk.h")).read()
     names = set(re.findall(r"\b(hpctopk_[a-z_]+)\s*\(", header))
     assert {"hpctopk_select", "hpctopk_workspace_bytes", "hpctopk_read_stats", "hpctopk_read_row_info",
-            "hpctopk_query_policy", "hpctopk_kernels_per_call", "hpctopk_status_string",
+            "hpctopk_query_policy", "hpctopk_kernels_per_call", "hpctopk_status_string", "hpctopk_select_padded",
             "hpctopk_version"} <= names
     for n in names:
         assert hasattr(lib, n), n
@@ -67,5 +67,11 @@ def test_argument_validation_returns_before_any_cuda_call(lib):
     assert f(ok_ptr, ok_ptr, ok_ptr, 4, 8, None, None, ok_ptr, None) == 1
     assert f(ok_ptr + 4, ok_ptr, ok_ptr, 4, 8, ok_ptr, None, ok_ptr, None) == 3      # scores not 16 B aligned
     assert f(ok_ptr, ok_ptr, ok_ptr, 4, 8, ok_ptr, None, ok_ptr + 16, None) == 3     # workspace not 256 B aligned
+    assert f(ok_ptr, None, ok_ptr, 4, 8, ok_ptr, None, ok_ptr, None) == 1               # packed form needs row_starts
+    g = lib.hpctopk_select_padded
+    assert g(ok_ptr, 64, ok_ptr, 0, 8, ok_ptr, None, ok_ptr, None) == 0
+    assert g(ok_ptr, -1, ok_ptr, 4, 8, ok_ptr, None, ok_ptr, None) == 1                 # negative pitch
+    assert g(ok_ptr, 64, None, 4, 8, ok_ptr, None, ok_ptr, None) == 1
+    assert g(ok_ptr + 4, 64, ok_ptr, 4, 8, ok_ptr, None, ok_ptr, None) == 3
     st = B.Stats()
     assert lib.hpctopk_read_stats(None, ctypes.byref(st), None) == 1

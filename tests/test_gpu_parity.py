@@ -194,3 +194,58 @@ def test_stage_timing_reports_the_dominant_kernel():
         B.hpctopk_stage_timing(False)
     assert calls == 3 and 0.0 < ms < 1000.0
     assert B.hpctopk_read_stage_timing() == (0.0, 0)
+
+
+@pytest.mark.parametrize("M,pitch,K", [(40, 70000, 2048), (40, 69999, 512), (600, 26000, 1024), (600, 25999, 2048)])
+def test_padded_matrix_entry_point_matches_the_packed_one_and_the_oracle(M, pitch, K):
+    """The paper's own layout (Section 2.1): M rows of a common pitch with valid lengths.  Aligned
+    and odd pitch, few rows (single kernel, KV-split) and many (three kernels); the padding holds
+    large values that must never be selected."""
+    g = torch.Generator(device=DEV).manual_seed(4000 + M + pitch)
+    X = torch.randn((M, pitch), generator=g, device=DEV, dtype=torch.float32)
+    rng = np.random.default_rng(M * 7 + pitch)
+    lengths = rng.integers(1, pitch + 1, size=M).astype(np.int32)
+    lengths[:3] = [pitch, 0, K]                              # full row, empty row, exactly K
+    cols = torch.arange(pitch, device=DEV)[None, :]
+    d_len = torch.from_numpy(lengths).to(DEV)
+    X = torch.where(cols < d_len[:, None], X, torch.full_like(X, 1e30))
+    out_idx, out_val, ws = B.hpctopk_select_padded(X, d_len, K)
+    torch.cuda.synchronize()
+    from oracle import native
+    from tests.helpers import assert_rows_match
+    scores = X.flatten().cpu().numpy()
+    starts = (np.arange(M, dtype=np.int64) * pitch).astype(np.int32)
+    want, _, _ = native.topk_stable_sort(scores, starts, lengths, K)
+    assert_rows_match(scores, starts, lengths, K, out_idx.cpu().numpy(), out_val.cpu().numpy(), want)
+    assert B.hpctopk_read_stats(ws)["error_flags"] == 0
+    # the packed entry point on the same memory gives the same sets
+    idx2, _, _ = B.hpctopk_select(X.flatten(), torch.from_numpy(starts).to(DEV), d_len, K)
+    torch.cuda.synchronize()
+    assert np.array_equal(np.sort(out_idx.cpu().numpy(), axis=1), np.sort(idx2.cpu().numpy(), axis=1))
+
+
+def test_padded_matrix_with_row_offsets_beyond_int32():
+    """r * pitch exceeds 2^31 elements: offsets are formed in 64 bits."""
+    M, pitch, K = 5, 600_000_000, 64
+    free, _ = torch.cuda.mem_get_info()
+    if free < 4 * (M - 1) * pitch + (8 << 30):
+        pytest.skip("not enough free device memory for a 9.6 GB matrix")
+    L = 100_000
+    X = torch.empty(((M - 1) * pitch + L,), device=DEV, dtype=torch.float32)     # last row holds only its valid part
+    g = torch.Generator(device=DEV).manual_seed(99)
+    rows = []
+    for r in range(M):
+        x = torch.randn(L, generator=g, device=DEV)
+        X[r * pitch: r * pitch + L] = x
+        rows.append(x.cpu().numpy())
+    d_len = torch.full((M,), L, dtype=torch.int32, device=DEV)
+    view = torch.as_strided(X, (M, L), (pitch, 1))
+    out_idx, out_val, _ = B.hpctopk_select_padded(view, d_len, K)
+    torch.cuda.synchronize()
+    from oracle import native
+    from tests.helpers import assert_rows_match
+    scores = np.concatenate(rows)
+    starts = (np.arange(M) * L).astype(np.int32)
+    lengths = np.full(M, L, dtype=np.int32)
+    want, _, _ = native.topk_stable_sort(scores, starts, lengths, K)
+    assert_rows_match(scores, starts, lengths, K, out_idx.cpu().numpy(), out_val.cpu().numpy(), want)
