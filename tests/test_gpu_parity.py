@@ -249,3 +249,13 @@ def test_padded_matrix_with_row_offsets_beyond_int32():
     lengths = np.full(M, L, dtype=np.int32)
     want, _, _ = native.topk_stable_sort(scores, starts, lengths, K)
     assert_rows_match(scores, starts, lengths, K, out_idx.cpu().numpy(), out_val.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("K,max_len", [(4096, 60000), (100, 20000), (1, 9000), (777, 30000)])
+def test_three_kernel_call_at_other_ranks(K, max_len):
+    """More than 512 rows (boundary, pass and refinement kernels) at the largest K, at small and
+    odd K, with the per-row trace compared where the sampled path is taken."""
+    batch = W.config1(DEV, seed=300 + K, num_rows=560, max_len=max_len, K=K)
+    assert B.hpctopk_kernels_per_call(batch.num_rows) == 3
+    stats, _, _, _ = _common().check_batch(batch, K, check_trace=True)
+    assert stats["rows_split"] == 0
