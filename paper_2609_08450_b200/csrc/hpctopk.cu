@@ -1388,19 +1388,22 @@ __global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params
   __syncthreads();
   {
     const int row = P.row_end - 1 - (int)blockIdx.x;
+    // everything the row needs from global memory, requested together
+    const RowRec* rec = pipe_rec(P) + row;
+    const uint4 rq0 = __ldg(reinterpret_cast<const uint4*>(rec));
+    const uint4 rq1 = __ldg(reinterpret_cast<const uint4*>(rec) + 1);
+    const uint32_t cnt = __ldcg(&pipe_cnt(P)[row]);
     const int64_t g0 = row_start(P, row);
     const int64_t L = P.row_lengths[row];
-    const RowRec* rec = pipe_rec(P) + row;
-    const bool sampled = L > (int64_t)cap && __ldg(&rec->usable) != 0u;
+    const bool sampled = L > (int64_t)cap && rq1.y != 0u;
     if (!sampled) {
       CandCtx rc;                                        // staging area: the row's own global range
       rc.cap_s = 0u; rc.cap = cap; rc.spill = pipe_cand(P, row);
       process_row<THREADS, U>(P, row, rc);               // short, direct, or recovery of an unusable view
     } else {
       __syncthreads();
-      if (tid < 4) sh.cutd[tid] = __ldg(&rec->cutd[tid]);
-      const int tau_pack = __ldg(&rec->tau_pack);
-      const uint32_t cnt = __ldcg(&pipe_cnt(P)[row]);
+      if (tid == 0) { sh.cutd[0] = rq0.x; sh.cutd[1] = rq0.y; sh.cutd[2] = rq0.z; sh.cutd[3] = rq0.w; }
+      const int tau_pack = (int)rq1.x;
       const bool band2 = (cnt & kBand2Flag) != 0u;
       const uint32_t C1 = cnt & ~kBand2Flag;             // entries of A(tau_1), or of A(tau_2) with the flag
       if (tid == 0) { sh.cand_count = C1; sh.count0 = 0; }
