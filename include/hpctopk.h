@@ -146,6 +146,14 @@ int hpctopk_select_padded(const float* scores, int64_t pitch, const int32_t* row
                           int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
                           void* workspace, hpctopk_stream_t stream);
 
+/* Ablation aid (Section 6.4 varies the stride and the margins): replace the built-in policy for
+ * all later calls of this process by stride `stride` (a power of two, 1..1024; 1 makes the view the
+ * whole row, i.e. an exact proposal) and margins K~ = rho K, K~_1 = rho1 K given in permille
+ * (1000 <= rho <= rho1 <= 2500; rho1 == rho switches the nested boundary off).  (0, 0, 0) restores
+ * the built-in policy.  The selected sets do not depend on the policy; routes and counters do.
+ * Host only; not thread-safe; returns HPCTOPK_ERR_INVALID_ARG for values outside these ranges. */
+int hpctopk_set_policy(int32_t stride, int32_t rho_permille, int32_t rho1_permille);
+
 /* Measurement aid (no counterpart in the paper): device time of the dominant kernel of each
  * call - the pass kernel of a three-kernel call, the one kernel otherwise - taken with CUDA
  * events recorded on the call's stream right before and after that launch.

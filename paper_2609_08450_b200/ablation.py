@@ -1,0 +1,90 @@
+"""Policy sweep on synthetic rows: sampling stride and margins against hit rates, bytes and time.
+
+Follows the ablations of Section 6.4 (margin rho, stride s, nested boundary on/off, exact
+proposal) on seeded synthetic rows, using the library's own counters.  The selected sets never
+depend on the policy; every run is compared with the sets of the built-in policy.
+
+    python -m paper_2609_08450_b200.ablation [--rows 592] [--kind drift|normal] [--iters 5]
+
+Prints one markdown table.  Needs a CUDA device.
+"""
+import argparse
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+K = 2048
+
+
+def make_rows(kind, rows, device):
+    if kind == "drift":      # the prefill-chunk recipe: indexer-style scores with key drift (locality)
+        return W.config3(device, num_rows=rows, offset=131072 - rows - 1)
+    lengths = np.full(rows, 131072, dtype=np.int64)       # exchangeable rows: i.i.d. N(0, 1)
+    g = torch.Generator(device=device).manual_seed(W.BASE_SEED + 77)
+    scores = torch.randn(int(lengths.sum()), generator=g, device=device, dtype=torch.float32)
+    starts = np.concatenate([[0], np.cumsum(lengths)[:-1]])
+    return W.Batch("normal_131072", scores, torch.from_numpy(starts.astype(np.int32)).to(device),
+                   torch.from_numpy(lengths.astype(np.int32)).to(device))
+
+
+def run(batch, iters, out_idx, out_val, ws):
+    for _ in range(2):
+        B.hpctopk_select(batch.scores, batch.row_starts, batch.row_lengths, K, out_idx, out_val, ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        B.hpctopk_select(batch.scores, batch.row_starts, batch.row_lengths, K, out_idx, out_val, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters, B.hpctopk_read_stats(ws)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--rows", type=int, default=592)
+    ap.add_argument("--kind", choices=["drift", "normal"], default="drift")
+    ap.add_argument("--iters", type=int, default=5)
+    args = ap.parse_args()
+    dev = "cuda"
+    batch = make_rows(args.kind, args.rows, dev)
+    M = batch.num_rows
+    out_idx = torch.empty((M, K), dtype=torch.int32, device=dev)
+    out_val = torch.empty((M, K), dtype=torch.float32, device=dev)
+    ws = torch.empty(B.hpctopk_workspace_bytes(M, K), dtype=torch.uint8, device=dev)
+    B.hpctopk_set_policy()
+    run(batch, 1, out_idx, out_val, ws)
+    want = torch.sort(out_idx, dim=1).values.clone()
+
+    policies = [("built-in (s=128, 1.5 / 1.75)", None)]
+    for rho in (1.0, 1.1, 1.25, 1.5, 1.75, 2.0):
+        policies.append((f"s=128, rho={rho}, rho1={rho + 0.25}", (128, rho, rho + 0.25)))
+    policies.append(("s=128, rho=1.5, nested boundary off", (128, 1.5, 1.5)))
+    for s in (16, 32, 64, 256, 512):
+        policies.append((f"s={s}, rho=1.5, rho1=1.75", (s, 1.5, 1.75)))
+    policies.append(("s=1 (exact proposal), rho=1.0, rho1=1.0", (1, 1.0, 1.0)))
+
+    print(f"| policy ({args.kind} rows, {M} x ~{batch.total_elements // M} scores, K={K}) | primary | band | second band "
+          f"| recovery + overflow | mean tail | row-equivalent reads | ms per call |")
+    print("|---|---|---|---|---|---|---|---|")
+    for name, pol in policies:
+        if pol is None:
+            B.hpctopk_set_policy()
+        else:
+            B.hpctopk_set_policy(*pol)
+        ms, st = run(batch, args.iters, out_idx, out_val, ws)
+        assert torch.equal(torch.sort(out_idx, dim=1).values, want), name
+        n = max(M, 1)
+        fin = st["rows_primary"] + st["rows_band"] + st["rows_band2"]
+        print(f"| {name} | {100 * st['rows_primary'] / n:.2f} % | {100 * st['rows_band'] / n:.2f} % "
+              f"| {100 * st['rows_band2'] / n:.2f} % | {100 * (st['rows_recovery'] + st['rows_overflow']) / n:.2f} % "
+              f"| {st['candidates_sum'] / max(fin, 1):.0f} "
+              f"| {(st['elements_scanned'] + st['elements_sampled']) / max(st['elements_valid'], 1):.4f} | {ms:.3f} |")
+    B.hpctopk_set_policy()
+
+
+if __name__ == "__main__":
+    main()

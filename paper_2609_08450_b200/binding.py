@@ -59,6 +59,8 @@ def lib():
         L.hpctopk_workspace_bytes.argtypes = [i32, i32]
         L.hpctopk_workspace_bytes.restype = ctypes.c_size_t
         L.hpctopk_query_policy.argtypes = [i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.hpctopk_set_policy.argtypes = [i32, i32, i32]
+        L.hpctopk_set_policy.restype = ctypes.c_int
         L.hpctopk_stage_timing.argtypes = [ctypes.c_int]
         L.hpctopk_read_stage_timing.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
         L.hpctopk_kernels_per_call.argtypes = [i32]
@@ -108,6 +110,13 @@ def hpctopk_query_policy(K, L):
 def hpctopk_kernels_per_call(num_rows):
     """Kernels one hpctopk_select call of ``num_rows`` rows launches (1 or 3)."""
     return int(lib().hpctopk_kernels_per_call(int(num_rows)))
+
+
+def hpctopk_set_policy(stride=0, rho=0.0, rho1=0.0):
+    """Override stride and margins (as factors of K) for later calls; no arguments: built-in policy."""
+    st = lib().hpctopk_set_policy(int(stride), int(round(rho * 1000)), int(round(rho1 * 1000)))
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
 
 
 def hpctopk_stage_timing(enable):

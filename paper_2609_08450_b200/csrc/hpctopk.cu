@@ -744,7 +744,8 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
   {
     int q_hi = (P.K + 4 * s - 1) / (4 * s);                           // bracket: sample rank ceil(K/4s)
     if (q_hi < 1) q_hi = 1;
-    const uint32_t q2 = (uint32_t)((3 * P.K + s - 1) / s);             // second band: sample rank ceil(3K/s)
+    uint32_t q2 = (uint32_t)((3 * P.K + s - 1) / s);                   // second band: sample rank ceil(3K/s)
+    if (q2 <= (uint32_t)P.q1) q2 = (uint32_t)P.q1 + 1u;
     const uint32_t quota[4] = {(uint32_t)P.q0, (uint32_t)P.q1, (uint32_t)q_hi, q2};
     // The four sample ranks are all small (at most 3K/s of the n_view samples), so their bins lie
     // within a few dozen bins of the best occupied one: one warp walks the histogram upwards from
@@ -1555,6 +1556,10 @@ constexpr int kPassThreads = HPCTOPK_PASS_T;
 const auto kRefineKernel = pipe_refine_kernel<kRefineThreads, 2, HPCTOPK_REFINE_MINB>;
 const auto kBoundaryKernel = pipe_boundary_kernel<kBoundaryThreads>;
 
+// Policy override for ablation runs (hpctopk_set_policy); all zero: the built-in policy.
+struct PolicyOverride { int32_t stride = 0, rho = 0, rho1 = 0; };
+PolicyOverride g_policy;
+
 // Event pair for this call, or -1 when stage timing is off, full, or the stream is being captured.
 int timing_slot(DeviceInfo& di, cudaStream_t st) {
   if (!di.timing || di.timed >= kTimingSlots) return -1;
@@ -1566,6 +1571,14 @@ int timing_slot(DeviceInfo& di, cudaStream_t st) {
 }  // namespace
 
 extern "C" {
+
+int hpctopk_set_policy(int32_t stride, int32_t rho_permille, int32_t rho1_permille) {
+  if (stride == 0 && rho_permille == 0 && rho1_permille == 0) { g_policy = PolicyOverride(); return HPCTOPK_OK; }
+  if (stride < 1 || stride > 1024 || (stride & (stride - 1)) != 0) return HPCTOPK_ERR_INVALID_ARG;
+  if (rho_permille < 1000 || rho1_permille < rho_permille || rho1_permille > 2500) return HPCTOPK_ERR_INVALID_ARG;
+  g_policy.stride = stride; g_policy.rho = rho_permille; g_policy.rho1 = rho1_permille;
+  return HPCTOPK_OK;
+}
 
 int hpctopk_stage_timing(int enable) {
   int dev = 0;
@@ -1649,7 +1662,7 @@ int hpctopk_kernels_per_call(int32_t num_rows) {
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route) {
   if (K < 1) return HPCTOPK_ERR_INVALID_ARG;
   if (K > HPCTOPK_MAX_K) return HPCTOPK_ERR_UNSUPPORTED_K;
-  if (stride) *stride = stride_for(K);
+  if (stride) *stride = g_policy.stride ? g_policy.stride : stride_for(K);
   if (capacity) *capacity = capacity_for(K);
   if (route) *route = L <= K ? HPCTOPK_ROUTE_SHORT : (L <= capacity_for(K) ? HPCTOPK_ROUTE_DIRECT : HPCTOPK_ROUTE_PRIMARY);
   return HPCTOPK_OK;
@@ -1740,9 +1753,14 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
   P.ws = static_cast<unsigned char*>(workspace);
   P.cap = capacity_for(K);
   P.cap_s = class_cap_s(cls) < P.cap ? class_cap_s(cls) : P.cap;
-  P.stride = stride_for(K);
-  P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);      // ceil(1.5 K / s)
-  P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);      // ceil(1.75 K / s)
+  P.stride = g_policy.stride ? g_policy.stride : stride_for(K);
+  if (g_policy.stride) {                                   // ablation runs: margins in permille
+    P.q0 = (int32_t)(((int64_t)g_policy.rho * K + 1000ll * P.stride - 1) / (1000ll * P.stride));
+    P.q1 = (int32_t)(((int64_t)g_policy.rho1 * K + 1000ll * P.stride - 1) / (1000ll * P.stride));
+  } else {
+    P.q0 = (3 * K + 2 * P.stride - 1) / (2 * P.stride);    // ceil(1.5 K / s)
+    P.q1 = (7 * K + 4 * P.stride - 1) / (4 * P.stride);    // ceil(1.75 K / s)
+  }
   P.split_enabled = split ? 1 : 0;
   P.pipe_rec_off = P.pipe_cnt_off = P.pipe_cand_off = P.pipe_spill_off = 0;
   const size_t smem = smem_bytes_for(class_cap_s(cls), split);

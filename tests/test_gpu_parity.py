@@ -259,3 +259,22 @@ def test_three_kernel_call_at_other_ranks(K, max_len):
     assert B.hpctopk_kernels_per_call(batch.num_rows) == 3
     stats, _, _, _ = _common().check_batch(batch, K, check_trace=True)
     assert stats["rows_split"] == 0
+
+
+def test_policy_override_changes_routes_not_results():
+    """hpctopk_set_policy (ablation aid): other strides and margins, the nested boundary switched
+    off, and the exact proposal (stride 1) all return the oracle's sets."""
+    K = 1024
+    batch = W.config1(DEV, seed=808, num_rows=560, max_len=40000, K=K)
+    c = _common()
+    try:
+        for pol in [(16, 1.5, 1.75), (256, 1.0, 1.0), (128, 2.0, 2.5), (1, 1.0, 1.0), (1024, 1.25, 1.5)]:
+            B.hpctopk_set_policy(*pol)
+            assert B.hpctopk_query_policy(K, 10 ** 6)[0] == pol[0]
+            c.check_batch(batch, K)
+            c.check_batch(W.config1(DEV, seed=809, num_rows=9, max_len=300000, K=K), K)   # split mode
+    finally:
+        B.hpctopk_set_policy()
+    assert B.hpctopk_query_policy(K, 10 ** 6)[0] == 64
+    with pytest.raises(B.HpcTopkError):
+        B.hpctopk_set_policy(100, 1.5, 1.75)            # not a power of two
