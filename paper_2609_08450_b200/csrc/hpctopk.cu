@@ -21,6 +21,7 @@
 #include <stddef.h>
 #include <stdlib.h>
 #include <type_traits>
+#include <mutex>
 
 #include "../../include/hpctopk.h"
 
@@ -1513,6 +1514,7 @@ struct DeviceInfo {
   int pipe_stages = 3;                              // tuning: run only the first n kernels (HPCTOPK_PIPE_STAGES)
 };
 DeviceInfo g_dev[64];
+std::mutex g_setup_mutex;
 
 size_t smem_bytes_for(int cap_s, bool split) {
   size_t b = align_up(sizeof(Shared), 16) + (size_t)cap_s * 8;
@@ -1699,6 +1701,7 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HPCTOPK_ERR_CUDA;
   DeviceInfo& di = g_dev[dev];
   const bool split = num_rows <= kSplitRowsMax;
+  std::unique_lock<std::mutex> setup_lock(g_setup_mutex);      // first call per device: one thread sets up
   if (!di.ready) {
     if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HPCTOPK_ERR_CUDA;
     init_cut_table_kernel<<<kBins * 32 / 256, 256>>>();
@@ -1745,6 +1748,7 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
     }
     di.ready = true;
   }
+  setup_lock.unlock();
   const Variant& v = kVariants[variant_index(di.variant, split)];
   const int cls = cap_class(K);
   Params P;
