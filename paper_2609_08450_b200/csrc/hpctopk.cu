@@ -1553,7 +1553,10 @@ PipeLayout pipe_layout(int rows, int K) {
 #define HPCTOPK_PASS_T 512
 #define HPCTOPK_PASS_MINB 3
 #endif
-const auto kPassKernel = pipe_pass_kernel<HPCTOPK_PASS_T, 2, HPCTOPK_PASS_MINB>;
+#ifndef HPCTOPK_PASS_U
+#define HPCTOPK_PASS_U 2
+#endif
+const auto kPassKernel = pipe_pass_kernel<HPCTOPK_PASS_T, HPCTOPK_PASS_U, HPCTOPK_PASS_MINB>;
 constexpr int kPassThreads = HPCTOPK_PASS_T;
 const auto kRefineKernel = pipe_refine_kernel<kRefineThreads, 2, HPCTOPK_REFINE_MINB>;
 const auto kBoundaryKernel = pipe_boundary_kernel<kBoundaryThreads>;
