@@ -1783,7 +1783,10 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
     // Three launches on the caller's stream.  (Cutting the rows into chunks and overlapping the
     // boundary and refinement kernels of neighbouring chunks with the pass kernel on extra streams
     // was measured: no gain, the streaming CTAs leave no room on the SMs until they exit, and
-    // limiting them to two per SM costs the pass kernel more than the overlap returns.)
+    // limiting them to two per SM costs the pass kernel more than the overlap returns.  Letting
+    // the refinement kernel of one chunk share the SMs with the boundary kernel of the next,
+    // between two pass kernels, was measured too: every extra chunk costs about 85 us, because
+    // each pass kernel then drains and the next one ramps up.)
     P.row_begin = 0;
     P.row_end = num_rows;
     const size_t smem_pass = smem_bytes_for(class_cap_s(cls), false);
