@@ -2,8 +2,10 @@
  *
  * C ABI of the library built from paper_2609_08450_b200/csrc/.  Unless a comment
  * says "host", every pointer below is a DEVICE pointer owned by the caller.  The
- * library allocates nothing and keeps no per-call state; the only process-wide
- * state is a per-device cache of launch attributes filled on first use.
+ * library allocates no device memory and keeps no per-call state; its process-wide
+ * state is a per-device cache of launch attributes and an 8 KB bin-to-cutoff table,
+ * both filled on first use, and the optional switches of hpctopk_set_policy and
+ * hpctopk_stage_timing (the latter creates CUDA events when first switched on).
  *
  * The operation is the standalone selector of "Sample-Guided Exact Top-K Selection
  * for Long-Context Sparse Attention": the operator contract of Section 2.1, computed
