@@ -890,7 +890,7 @@ __device__ __noinline__ void helper_main(const Grp G, const Params& P, uint32_t 
   uint32_t* rowcnt = arrive + kSplitRowsMax;
   const size_t cand_off = align_up(kOffRowInfo + (size_t)P.num_rows * sizeof(hpctopk_row_info), 256);
   const Buf buf = make_slot_buf(P, s, rw, sw);
-  Task t;
+  Task t{};
   uint32_t uses = 0;                      // descriptors posted so far (mbarrier phase bookkeeping)
   // task claiming: one statically assigned task per group, then the device counter, one claim in flight
   const uint32_t n_static = gridDim.x * kSlots;
