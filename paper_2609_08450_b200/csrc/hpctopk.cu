@@ -1,17 +1,24 @@
 // hpctopk: exact Top-K over ragged FP32 score rows, hand-written for sm_100a.
 //
-// One persistent kernel.  CTAs claim tasks (a whole row, or one contiguous segment of a long
-// row) from a device counter; everything that depends on row lengths is decided on the device,
-// so the launch geometry is a function of (num_rows, K, device) only.
+// Two launch forms over the same device functions.  A single persistent kernel (hpctopk_kernel):
+// CTAs claim tasks (a whole row, or one contiguous segment of a long row) from a device counter;
+// used for calls of few rows, where long rows are split over CTAs, and for very many rows.  And a
+// three-kernel pipeline (pipe_boundary_kernel, pipe_pass_kernel, pipe_refine_kernel) for calls in
+// between, which keeps the kernel that reads every score streaming all the time.  Everything that
+// depends on row lengths is decided on the device, so the launch geometry is a function of
+// (num_rows, K, device) only.
 //
 // Per row (notation of Sections 4.2-4.4 of the paper):
 //   Phase 1  stride-s view -> 2048-bin coarse histogram (11 leading bits of the fp16 key) ->
-//            tau_0, tau_1 -> inclusive FP32 cutoffs (as ordered keys)
-//   Phase 2  one complete-row pass: key <= cutoff ? append (key, index) to shared memory,
-//            count C(tau_0), add to the leading-digit histogram
-//   Phase 3  radix refinement 11+11+10 over the admitted tail, continued over the index bits
-//            when the final equal-key group is larger than the remaining quota
-//   recovery band pass for tau_1; storage-free full-radix select over the whole row otherwise
+//            tau_0, nested tau_1 (plus a bracket bin and a wider tau_2 of the same histogram) ->
+//            inclusive FP32 cutoffs (as ordered keys)
+//   Phase 2  one complete-row pass: key <= cutoff(tau_1) ? append (key, index); C(tau_0) is
+//            counted from the stored tail, so the band extension costs no second pass
+//   Phase 3  one pass over a row-adaptive 2048-bin digit and a ranking of the boundary bin; the
+//            general radix refinement 11+11+10, continued over the index bits when the final
+//            equal-key group is larger than the remaining quota, behind it
+//   recovery one band pass for (tau_1, tau_2]; storage-free full-radix select over the whole row
+//            otherwise
 //
 // Keys: kd(x) is the descending sortable key (smaller key = larger score), kd = u for a set
 // sign bit and u ^ 0x7FFFFFFF otherwise, u the raw bits.
@@ -54,7 +61,7 @@ constexpr size_t kOffStats = 256;                    // hpctopk_stats (176 B)
 constexpr size_t kOffSplit = 512;                    // arrive[512], count[512], count of A(tau_0)[512]
 constexpr size_t kZeroBytes = kOffSplit + 3 * kSplitRowsMax * sizeof(uint32_t);
 constexpr size_t kOffRowInfo = 8192;
-constexpr int kPrefetchAheadBytes = 65536;   // L2 prefetch distance inside a row's scan
+constexpr int kPrefetchAheadBytes = 65536;   // L2 prefetch distance inside a row's scan (warp-specialised kernels)
 constexpr int kPrefetchHeadBytes = 131072;   // bytes of the next task's range warmed in L2 ahead of time
 constexpr int kMaxGrid = 1024;         // upper bound on resident CTAs (sizes the spill region)
 
