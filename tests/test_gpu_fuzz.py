@@ -1,0 +1,72 @@
+"""Randomised shapes against the stable-sort oracle: row counts on both sides of the call-shape
+limits, any K, rows at odd offsets with gaps between them, negative lengths, structured and
+heavy-tailed values with infinities and signed zeros.  Seeds are fixed; every case is small."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import native
+from paper_2609_08450_b200 import binding as B, build, workloads as W
+from tests.helpers import assert_rows_match
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+build.build()
+
+
+def _case(rng):
+    K = int(rng.choice([1, 2, 3, 7, 64, 100, 511, 512, 1000, 1024, 2047, 2048, 3000, 4096]))
+    M = int(rng.choice([1, 2, 5, 17, 64, 200, 512, 513, 600, 900]))
+    stride, cap, _ = B.hpctopk_query_policy(K, 10 ** 6)
+    mode = int(rng.integers(0, 4))
+    maxlen = int(rng.choice([50, 3000, cap + 10, 3 * cap, 40000, 150000]))
+    rows, total = [], 0
+    for _ in range(M):
+        L = int(rng.integers(0, maxlen + 1))
+        if rng.random() < 0.05:
+            L = int(rng.choice([0, 1, max(K - 1, 1), K, K + 1, cap, cap + 1]))
+        if total + L > 3_000_000:
+            L = min(L, 1000)
+        total += L
+        if L == 0:
+            rows.append(np.zeros(0, np.float32))
+        elif mode == 0:
+            rows.append(rng.normal(size=L).astype(np.float32))
+        elif mode == 1:
+            kind = W.ADVERSARIAL_KINDS[int(rng.integers(0, len(W.ADVERSARIAL_KINDS)))]
+            rows.append(np.ascontiguousarray(W.adversarial_row(kind, L, K, stride, rng), dtype=np.float32))
+        elif mode == 2:
+            levels = int(rng.choice([2, 5, 50, 1000]))
+            scale = np.float32(rng.choice([1.0, -1.0, 1e-30, 1e30]))
+            rows.append(rng.integers(0, levels, size=L).astype(np.float32) * scale)
+        else:
+            x = rng.standard_t(3, size=L).astype(np.float32)
+            x[rng.random(L) < 0.01] = np.float32(rng.choice([np.inf, -np.inf, 0.0, -0.0]))
+            rows.append(x)
+    lengths = np.array([len(x) for x in rows], dtype=np.int32)
+    if M > 1 and rng.random() < 0.3:
+        lengths[int(rng.integers(0, M))] = -int(rng.integers(1, 5))
+    gaps = rng.integers(0, 4, size=M)
+    starts, parts, pos = np.zeros(M, dtype=np.int32), [], 0
+    for r in range(M):
+        parts.append(np.full(int(gaps[r]), np.float32(9e30), np.float32))
+        pos += int(gaps[r])
+        starts[r] = pos
+        parts.append(rows[r])
+        pos += len(rows[r])
+    scores = np.concatenate(parts + [np.zeros(4, np.float32)])
+    return K, scores, starts, lengths, rng.random() < 0.8
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_match_the_oracle(seed):
+    rng = np.random.default_rng(7000 + seed)
+    for _ in range(12):
+        K, scores, starts, lengths, want_values = _case(rng)
+        out_idx, out_val, ws = B.hpctopk_select(torch.from_numpy(scores).to(DEV), torch.from_numpy(starts).to(DEV),
+                                                torch.from_numpy(lengths).to(DEV), K, want_values=want_values)
+        torch.cuda.synchronize()
+        want, _, _ = native.topk_stable_sort(scores, starts, lengths, K)
+        assert_rows_match(scores, starts, lengths, K, out_idx.cpu().numpy(),
+                          out_val.cpu().numpy() if out_val is not None else None, want)
+        assert B.hpctopk_read_stats(ws)["error_flags"] == 0
