@@ -148,6 +148,17 @@ int hpctopk_select_padded(const float* scores, int64_t pitch, const int32_t* row
                           int32_t num_rows, int32_t K, int32_t* out_idx, float* out_val,
                           void* workspace, hpctopk_stream_t stream);
 
+/* Optional ordered output (the contract of Section 2.1 imposes no slot order; consumers that
+ * want one call this after a select on the same stream).  Sorts the K slots of every row of
+ * out_idx / out_val in place by score descending - under the monotone key, so -0.0 follows +0.0 -
+ * and index ascending among equal scores; -1 sentinels stay last.  `out_val` may be NULL, in which
+ * case the scores are read through `scores` and `row_starts` (or `pitch` when row_starts is NULL,
+ * as in hpctopk_select_padded); with `out_val` given, `scores` and `row_starts` are not read and
+ * may be NULL.  One kernel, no workspace.  Returns HPCTOPK_ERR_INVALID_ARG / _UNSUPPORTED_K as
+ * the selector does. */
+int hpctopk_sort_output(const float* scores, const int32_t* row_starts, int64_t pitch, int32_t num_rows,
+                        int32_t K, int32_t* out_idx, float* out_val, hpctopk_stream_t stream);
+
 /* Ablation aid (Section 6.4 varies the stride and the margins): replace the built-in policy for
  * all later calls of this process by stride `stride` (a power of two, 1..1024; 1 makes the view the
  * whole row, i.e. an exact proposal) and margins K~ = rho K, K~_1 = rho1 K given in permille

@@ -59,6 +59,8 @@ def lib():
         L.hpctopk_workspace_bytes.argtypes = [i32, i32]
         L.hpctopk_workspace_bytes.restype = ctypes.c_size_t
         L.hpctopk_query_policy.argtypes = [i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.hpctopk_sort_output.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp]
+        L.hpctopk_sort_output.restype = ctypes.c_int
         L.hpctopk_set_policy.argtypes = [i32, i32, i32]
         L.hpctopk_set_policy.restype = ctypes.c_int
         L.hpctopk_stage_timing.argtypes = [ctypes.c_int]
@@ -110,6 +112,21 @@ def hpctopk_query_policy(K, L):
 def hpctopk_kernels_per_call(num_rows):
     """Kernels one hpctopk_select call of ``num_rows`` rows launches (1 or 3)."""
     return int(lib().hpctopk_kernels_per_call(int(num_rows)))
+
+
+def hpctopk_sort_output(out_idx, out_val=None, scores=None, row_starts=None, pitch=0, stream=None):
+    """Sort each row of (out_idx, out_val) in place: score descending, index ascending on ties."""
+    import torch
+    M, K = int(out_idx.size(0)), int(out_idx.size(1))
+    if stream is None:
+        stream = torch.cuda.current_stream(out_idx.device)
+    with torch.cuda.device(out_idx.device):
+        st = int(lib().hpctopk_sort_output(scores.data_ptr() if scores is not None else None,
+                                           row_starts.data_ptr() if row_starts is not None else None, int(pitch), M, K,
+                                           out_idx.data_ptr(), out_val.data_ptr() if out_val is not None else None,
+                                           stream.cuda_stream))
+    if st != HPCTOPK_OK:
+        raise HpcTopkError(st)
 
 
 def hpctopk_set_policy(stride=0, rho=0.0, rho1=0.0):

@@ -1457,6 +1457,55 @@ __global__ void __launch_bounds__(THREADS, MINB) pipe_refine_kernel(const Params
   if (tid == 0) stats_flush(P.ws);
 }
 
+
+// ---------------------------------------------------------------- ordered output (optional)
+// Sorts the K slots of every row in place by (score descending under the key, index ascending);
+// sentinel slots stay last.  One CTA per row, bitonic sort of 64-bit composites (kd << 32 | idx)
+// in shared memory (N = smallest power of two >= K, at most 4096 entries = 32 KB).
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) sort_rows_kernel(const Params P) {
+  extern __shared__ __align__(16) unsigned char sort_smem[];
+  unsigned long long* a = reinterpret_cast<unsigned long long*>(sort_smem);
+  const int row = blockIdx.x;
+  const uint32_t K = (uint32_t)P.K;
+  uint32_t N = 1;
+  while (N < K) N <<= 1;
+  const int64_t g0 = row_start(P, row);
+  int32_t* oi = P.out_idx + (int64_t)row * P.K;
+  float* ov = P.out_val ? P.out_val + (int64_t)row * P.K : nullptr;
+  for (uint32_t i = threadIdx.x; i < N; i += THREADS) {
+    unsigned long long v = ~0ull;                                  // sentinel and padding slots sort last
+    if (i < K) {
+      const int32_t idx = oi[i];
+      if (idx >= 0) {
+        const uint32_t u = __float_as_uint(ov ? ov[i] : __ldg(P.scores + g0 + idx));
+        v = ((unsigned long long)kd_of_bits(u) << 32) | (uint32_t)idx;
+      }
+    }
+    a[i] = v;
+  }
+  __syncthreads();
+  for (uint32_t k = 2; k <= N; k <<= 1) {
+    for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+      for (uint32_t i = threadIdx.x; i < N; i += THREADS) {
+        const uint32_t l = i ^ j;
+        if (l > i) {
+          const unsigned long long x = a[i], y = a[l];
+          const bool up = (i & k) == 0;
+          if ((x > y) == up) { a[i] = y; a[l] = x; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  for (uint32_t i = threadIdx.x; i < K; i += THREADS) {
+    const unsigned long long v = a[i];
+    const bool valid = v != ~0ull;
+    oi[i] = valid ? (int32_t)(uint32_t)v : -1;
+    if (ov) ov[i] = valid ? __uint_as_float(bits_of_kd((uint32_t)(v >> 32))) : __uint_as_float(0xFF800000u);
+  }
+}
+
 }  // namespace
 #include "hpctopk_ws.cuh"            // namespace wsk: scanner warps + helper groups
 #define HPCTOPK_WS_NAMESPACE wsf     // namespace wsf: single-role variant, warp-synchronous compaction
@@ -1833,6 +1882,25 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
     v.fn<<<grid, v.threads, smem, st>>>(P);
     if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
   }
+  if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
+  return HPCTOPK_OK;
+}
+
+int hpctopk_sort_output(const float* scores, const int32_t* row_starts, int64_t pitch, int32_t num_rows, int32_t K,
+                        int32_t* out_idx, float* out_val, hpctopk_stream_t stream) {
+  if (num_rows < 0 || K < 1 || pitch < 0) return HPCTOPK_ERR_INVALID_ARG;
+  if (K > HPCTOPK_MAX_K) return HPCTOPK_ERR_UNSUPPORTED_K;
+  if (num_rows == 0) return HPCTOPK_OK;
+  if (!out_idx || (!out_val && !scores)) return HPCTOPK_ERR_INVALID_ARG;
+  Params P;
+  P.scores = scores; P.row_starts = row_starts; P.pitch = pitch; P.row_lengths = nullptr;
+  P.num_rows = num_rows; P.K = K; P.out_idx = out_idx; P.out_val = out_val; P.ws = nullptr;
+  P.cap = P.cap_s = 0; P.stride = 1; P.q0 = P.q1 = 0; P.split_enabled = 0;
+  P.pipe_rec_off = P.pipe_cnt_off = P.pipe_cand_off = P.pipe_spill_off = 0;
+  P.row_begin = 0; P.row_end = num_rows;
+  size_t n = 1;
+  while (n < (size_t)K) n <<= 1;
+  sort_rows_kernel<512><<<num_rows, 512, n * sizeof(unsigned long long), reinterpret_cast<cudaStream_t>(stream)>>>(P);
   if (cudaGetLastError() != cudaSuccess) return HPCTOPK_ERR_CUDA;
   return HPCTOPK_OK;
 }

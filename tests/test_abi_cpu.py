@@ -22,7 +22,7 @@ def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "hpctopk.h")).read()
     names = set(re.findall(r"\b(hpctopk_[a-z_]+)\s*\(", header))
     assert {"hpctopk_select", "hpctopk_workspace_bytes", "hpctopk_read_stats", "hpctopk_read_row_info",
-            "hpctopk_query_policy", "hpctopk_kernels_per_call", "hpctopk_status_string", "hpctopk_select_padded", "hpctopk_set_policy", "hpctopk_stage_timing",
+            "hpctopk_query_policy", "hpctopk_kernels_per_call", "hpctopk_status_string", "hpctopk_select_padded", "hpctopk_sort_output", "hpctopk_set_policy", "hpctopk_stage_timing",
             "hpctopk_version"} <= names
     for n in names:
         assert hasattr(lib, n), n

@@ -297,3 +297,28 @@ def test_many_small_rows_at_the_call_shape_limits(M):
     assert B.hpctopk_kernels_per_call(M) == (3 if M <= 8192 else 1)
     stats, _, _, _ = _common().check_batch(batch, K, check_trace=True)
     assert stats["rows_short"] > 0 and stats["rows_direct"] > 0 and stats["rows_primary"] > 0
+
+
+@pytest.mark.parametrize("K", [1, 100, 2048, 4096])
+def test_sort_output_gives_the_oracle_order(K):
+    """hpctopk_sort_output: slots in the order of the definition (score descending under the key,
+    lower index first among equal scores), sentinels last; with values, and with indices only."""
+    stride, cap, _ = B.hpctopk_query_policy(K, 10 ** 6)
+    rng = np.random.default_rng(K)
+    rows = [rng.normal(size=int(L)).astype(np.float32) for L in rng.integers(0, 3 * cap, size=24)]
+    for kind in ("levels16", "signed_zeros", "constant", "neg_inf_pad"):
+        if kind in W.ADVERSARIAL_KINDS:
+            rows.append(np.ascontiguousarray(W.adversarial_row(kind, 2 * cap + 5, K, stride, rng), dtype=np.float32))
+    rows.append(np.array([0.0, -0.0, 0.0, -0.0, 1.0, -np.inf, np.inf, 1.0], dtype=np.float32))
+    batch = _batch_from_rows(rows, "sort_output")
+    scores, starts, lengths = batch.host()
+    from oracle import native
+    want_idx, want_val, _ = native.topk_stable_sort(scores, starts, lengths, K)
+    for with_values in (True, False):
+        out_idx, out_val, _ = B.hpctopk_select(batch.scores, batch.row_starts, batch.row_lengths, K,
+                                               want_values=with_values)
+        B.hpctopk_sort_output(out_idx, out_val, scores=batch.scores, row_starts=batch.row_starts)
+        torch.cuda.synchronize()
+        assert np.array_equal(out_idx.cpu().numpy(), want_idx)
+        if with_values:
+            assert np.array_equal(out_val.cpu().numpy().view(np.uint32), want_val.view(np.uint32))
