@@ -1487,13 +1487,12 @@ __global__ void __launch_bounds__(THREADS) sort_rows_kernel(const Params P) {
   __syncthreads();
   for (uint32_t k = 2; k <= N; k <<= 1) {
     for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-      for (uint32_t i = threadIdx.x; i < N; i += THREADS) {
-        const uint32_t l = i ^ j;
-        if (l > i) {
-          const unsigned long long x = a[i], y = a[l];
-          const bool up = (i & k) == 0;
-          if ((x > y) == up) { a[i] = y; a[l] = x; }
-        }
+      for (uint32_t p = threadIdx.x; p < (N >> 1); p += THREADS) {     // one compare-exchange per pair
+        const uint32_t i = ((p & ~(j - 1u)) << 1) | (p & (j - 1u));       // j is a power of two
+        const uint32_t l = i | j;
+        const unsigned long long x = a[i], y = a[l];
+        const bool up = (i & k) == 0;
+        if ((x > y) == up) { a[i] = y; a[l] = x; }
       }
       __syncthreads();
     }
