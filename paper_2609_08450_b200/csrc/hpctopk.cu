@@ -119,7 +119,7 @@ __device__ __forceinline__ int64_t row_start(const Params& P, int row) {
 
 struct Shared {
   hpctopk_stats acc;         // this CTA's counters (first member of every kernel's shared state)
-  uint32_t hist[kBins];
+  alignas(16) uint32_t hist[kBins];   // read and cleared as 16-byte vectors
   uint32_t warp_sums[32];
   uint32_t cand_count;
   uint32_t out_count;
@@ -403,7 +403,8 @@ __device__ __forceinline__ void locate_n(const uint32_t (&quota)[N]) {
 
 template <int THREADS>
 __device__ __forceinline__ void clear_hist(Shared& sh) {
-  for (int b = threadIdx.x; b < kBins; b += THREADS) sh.hist[b] = 0;
+  uint4* hv = reinterpret_cast<uint4*>(sh.hist);
+  for (int b = threadIdx.x; b < kBins / 4; b += THREADS) hv[b] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // Admission test on raw bits, one integer compare per score (Section 5.3 compares the FP32
@@ -933,8 +934,16 @@ __device__ __noinline__ bool select_adaptive(const CandCtx cc, uint32_t C, uint3
   }
   __syncthreads();
   if (STAGE_OUT) {
-    for (uint32_t i = tid; i < K; i += THREADS) out_idx[i] = w_idx[i];
-    if (out_val) for (uint32_t i = tid; i < K; i += THREADS) out_val[i] = w_val[i];
+    const bool vec = (K & 3u) == 0u && ((reinterpret_cast<uintptr_t>(out_idx) | reinterpret_cast<uintptr_t>(out_val)) & 15u) == 0u;
+    if (vec) {                                   // whole 16-byte vectors (K words each of indices and values)
+      const uint4* si = reinterpret_cast<const uint4*>(w_idx);
+      const uint4* sv = reinterpret_cast<const uint4*>(w_val);
+      for (uint32_t i = tid; i < (K >> 2); i += THREADS) reinterpret_cast<uint4*>(out_idx)[i] = si[i];
+      if (out_val) for (uint32_t i = tid; i < (K >> 2); i += THREADS) reinterpret_cast<uint4*>(out_val)[i] = sv[i];
+    } else {
+      for (uint32_t i = tid; i < K; i += THREADS) out_idx[i] = w_idx[i];
+      if (out_val) for (uint32_t i = tid; i < K; i += THREADS) out_val[i] = w_val[i];
+    }
   }
   DSTAMP(4, ts);
   return true;
