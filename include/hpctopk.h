@@ -88,8 +88,9 @@ const char* hpctopk_status_string(int status);
 
 /* Bytes of device workspace hpctopk_select needs for up to `max_num_rows` rows at rank K.
  * Independent of row width (Section 2.1, "Deployment requirements"): a constant plus 16 bytes
- * per row, plus - for calls of 513 to 8192 rows, which run as three kernels - one candidate
- * range of max(4K, 4096) 8-byte entries per row (64 KB per row at K = 2048).  Host only.
+ * per row, plus - for calls of more than 512 rows, which run as three kernels per 8192 rows -
+ * one candidate range of max(4K, 4096) 8-byte entries for each of up to 8192 rows (64 KB per row
+ * at K = 2048).  Host only.
  * Returns 0 for invalid arguments. */
 size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K);
 
@@ -103,8 +104,8 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K);
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route);
 
 /* Number of kernels one hpctopk_select call of `num_rows` rows launches on the current device
- * (1: the single persistent kernel; 3: boundary, pass and refinement kernels, calls of 513 to
- * 8192 rows).  Host only;
+ * (1: the single persistent kernel, calls of at most 512 rows; otherwise 3 - boundary, pass
+ * and refinement kernel - for every 8192 rows).  Host only;
  * returns 0 for num_rows <= 0. */
 int hpctopk_kernels_per_call(int32_t num_rows);
 
@@ -126,8 +127,8 @@ int hpctopk_kernels_per_call(int32_t num_rows);
  *   workspace   >= hpctopk_workspace_bytes(num_rows, K) bytes, 256-byte aligned; contents
  *               need not be initialised; calls that may overlap on the device need
  *               distinct workspaces
- *   stream      all work is enqueued on `stream` (one small memset and one or three kernels
- *               whose launch geometry depends only on num_rows, K and the device); nothing
+ *   stream      all work is enqueued on `stream` (one small memset and one kernel, or three
+ *               per 8192 rows, whose launch geometry depends only on num_rows, K and the device); nothing
  *               is read back, so the call can be captured in a CUDA graph and replayed with
  *               new contents in the same buffers.  The very first call on a device also
  *               fills a 8 KB lookup table and synchronises the device once: make it
@@ -172,9 +173,10 @@ int hpctopk_set_policy(int32_t stride, int32_t rho_permille, int32_t rho1_permil
  * events recorded on the call's stream right before and after that launch.
  *   hpctopk_stage_timing(1) creates the events for the current device (first use) and switches
  *   the recording on, hpctopk_stage_timing(0) switches it off.  Calls made while the stream is
- *   being captured are not timed.  At most 1024 calls are kept between two reads.
+ *   being captured are not timed.  At most 1024 launches are kept between two reads.
  *   hpctopk_read_stage_timing waits for the recorded events, returns the summed milliseconds
- *   and the number of calls they cover, and starts a new interval.  Host only; not thread-safe. */
+ *   (over every launch of that kernel) and the number of calls they cover, and starts a new
+ *   interval.  Host only; not thread-safe. */
 int hpctopk_stage_timing(int enable);
 int hpctopk_read_stage_timing(float* total_ms, int32_t* calls);
 

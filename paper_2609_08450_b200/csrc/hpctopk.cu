@@ -2,9 +2,9 @@
 //
 // Two launch forms over the same device functions.  A single persistent kernel (hpctopk_kernel):
 // CTAs claim tasks (a whole row, or one contiguous segment of a long row) from a device counter;
-// used for calls of few rows, where long rows are split over CTAs, and for very many rows.  And a
-// three-kernel pipeline (pipe_boundary_kernel, pipe_pass_kernel, pipe_refine_kernel) for calls in
-// between, which keeps the kernel that reads every score streaming all the time.  Everything that
+// used for calls of few rows, where long rows are split over CTAs.  And a three-kernel pipeline
+// (pipe_boundary_kernel, pipe_pass_kernel, pipe_refine_kernel) for all other calls, which keeps
+// the kernel that reads every score streaming all the time.  Everything that
 // depends on row lengths is decided on the device, so the launch geometry is a function of
 // (num_rows, K, device) only.
 //
@@ -802,7 +802,9 @@ __device__ __noinline__ bool phase1(const Params& P, int row, int64_t g0, int64_
 
 // The row's boundary: read from the record a boundary kernel left (when the call ran one), else
 // computed here.  Leaves the cutoffs in sh.cutd like phase1; contains block barriers.
-__device__ __forceinline__ RowRec* pipe_rec(const Params& P) { return reinterpret_cast<RowRec*>(P.ws + P.pipe_rec_off); }
+// The per-row regions of the pipeline's workspace are indexed from the first row of the launch
+// (a call of very many rows runs as several launches that reuse them).
+__device__ __forceinline__ RowRec* pipe_rec(const Params& P) { return reinterpret_cast<RowRec*>(P.ws + P.pipe_rec_off) - P.row_begin; }
 template <int THREADS>
 __device__ __forceinline__ bool row_boundary(const Params& P, int row, int64_t g0, int64_t L, int& tau_pack) {
   if (P.pipe_rec_off == 0) return phase1<THREADS>(P, row, g0, L, tau_pack);
@@ -1305,9 +1307,9 @@ __global__ void __launch_bounds__(THREADS, MINB) hpctopk_kernel(const Params P) 
 // time and the short phases run at their own, higher occupancy.  Cost: the admitted tails cross
 // HBM once each way (about 57 KB per row at K = 2048, 11 % of a 129 K-score row).
 constexpr uint32_t kBand2Flag = 0x80000000u;    // in a row's admitted count: the tail includes the second band
-__device__ __forceinline__ uint32_t* pipe_cnt(const Params& P) { return reinterpret_cast<uint32_t*>(P.ws + P.pipe_cnt_off); }
+__device__ __forceinline__ uint32_t* pipe_cnt(const Params& P) { return reinterpret_cast<uint32_t*>(P.ws + P.pipe_cnt_off) - P.row_begin; }
 __device__ __forceinline__ uint2* pipe_cand(const Params& P, int row) {
-  return reinterpret_cast<uint2*>(P.ws + P.pipe_cand_off) + (size_t)row * (size_t)P.cap;
+  return reinterpret_cast<uint2*>(P.ws + P.pipe_cand_off) + (size_t)(row - P.row_begin) * (size_t)P.cap;
 }
 
 template <int THREADS>
@@ -1553,8 +1555,8 @@ const Variant kVariants[] = {
 };
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 // 0 selects the warp-specialised kernel, v >= 1 the single-role kernel kVariants[v - 1].
-// kPipeVariant selects the three-kernel pipeline (calls of at most kPipeRowsMax rows; larger calls
-// use the single kernel, whose workspace does not grow with the row count).
+// kPipeVariant selects the three-kernel pipeline for calls beyond the split-mode row count, one
+// launch of the three per kPipeRowsMax rows (the per-row workspace regions are sized for that many).
 constexpr int kPipeVariant = 200;
 constexpr int kDefaultVariant = kPipeVariant;
 constexpr int kMonoVariant = 4;
@@ -1577,6 +1579,7 @@ struct DeviceInfo {
   int boundary_per_sm = 0;                          // pipeline: boundary kernel
   bool timing = false;                              // hpctopk_stage_timing
   int timed = 0;                                    // event pairs recorded since the last read
+  int timed_calls = 0;                              // calls they belong to (a call of many rows records several)
   cudaEvent_t ev0[kTimingSlots] = {}, ev1[kTimingSlots] = {};
   int pipe_stages = 3;                              // tuning: run only the first n kernels (HPCTOPK_PIPE_STAGES)
 };
@@ -1606,10 +1609,11 @@ int class_cap_s(int cls) { return smem_capacity_for(cls == 0 ? 1024 : (cls == 1 
 // `capacity` entries per row (a pass CTA writes what exceeds its shared memory straight into
 // that range, and the refinement kernel stages nothing on chip, so there are no overflow slices).
 struct PipeLayout { size_t rec, cnt, cand, total; };
-PipeLayout pipe_layout(int rows, int K) {
+PipeLayout pipe_layout(int all_rows, int K) {
   const size_t cap = (size_t)capacity_for(K);
+  const int rows = all_rows < kPipeRowsMax ? all_rows : kPipeRowsMax;      // rows of one launch
   PipeLayout l;
-  l.rec = align_up(kOffRowInfo + (size_t)rows * sizeof(hpctopk_row_info), 256);
+  l.rec = align_up(kOffRowInfo + (size_t)all_rows * sizeof(hpctopk_row_info), 256);
   l.cnt = align_up(l.rec + (size_t)rows * sizeof(RowRec), 256);
   l.cand = align_up(l.cnt + (size_t)rows * sizeof(uint32_t), 256);
   l.total = align_up(l.cand + (size_t)rows * cap * 8, 256);
@@ -1682,8 +1686,9 @@ int hpctopk_read_stage_timing(float* total_ms, int32_t* calls) {
     sum += ms;
   }
   *total_ms = sum;
-  *calls = di.timed;
+  *calls = di.timed_calls;
   di.timed = 0;
+  di.timed_calls = 0;
   return HPCTOPK_OK;
 }
 
@@ -1717,7 +1722,7 @@ size_t hpctopk_workspace_bytes(int32_t max_num_rows, int32_t K) {
   if (spill_wf > spill) spill = spill_wf;
   b += spill;
   b = align_up(b, 256);
-  if (max_num_rows <= kPipeRowsMax) {
+  {
     const size_t p = pipe_layout(max_num_rows, K).total;
     if (p > b) b = p;
   }
@@ -1728,7 +1733,8 @@ int hpctopk_kernels_per_call(int32_t num_rows) {
   if (num_rows <= 0) return 0;
   const char* env = getenv("HPCTOPK_VARIANT");
   const int variant = env ? atoi(env) : kDefaultVariant;
-  return (variant == kPipeVariant && num_rows > kSplitRowsMax && num_rows <= kPipeRowsMax) ? 3 : 1;
+  if (variant != kPipeVariant || num_rows <= kSplitRowsMax) return 1;
+  return 3 * ((num_rows + kPipeRowsMax - 1) / kPipeRowsMax);
 }
 
 int hpctopk_query_policy(int32_t K, int64_t L, int32_t* stride, int32_t* capacity, int32_t* route) {
@@ -1843,7 +1849,7 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(workspace, 0, kZeroBytes, st) != cudaSuccess) { cudaGetLastError(); return HPCTOPK_ERR_CUDA; }
   // Calls of few rows (split mode) are latency-bound: one launch and on-chip tails serve them better.
-  if (di.variant == kPipeVariant && num_rows <= kPipeRowsMax && !split) {
+  if (di.variant == kPipeVariant && !split) {
     const PipeLayout l = pipe_layout(num_rows, K);
     P.pipe_rec_off = (int64_t)l.rec; P.pipe_cnt_off = (int64_t)l.cnt;
     P.pipe_cand_off = (int64_t)l.cand;
@@ -1854,20 +1860,29 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
     // the refinement kernel of one chunk share the SMs with the boundary kernel of the next,
     // between two pass kernels, was measured too: every extra chunk costs about 85 us, because
     // each pass kernel then drains and the next one ramps up.)
-    P.row_begin = 0;
-    P.row_end = num_rows;
     const size_t smem_pass = smem_bytes_for(class_cap_s(cls), false);
     const size_t smem_small = smem_bytes_for(0, false);
-    int g1 = di.sm_count * di.boundary_per_sm;
-    if (g1 > num_rows) g1 = num_rows;
-    kBoundaryKernel<<<g1, kBoundaryThreads, smem_small, st>>>(P);
-    const int slot = timing_slot(di, st);
-    if (slot >= 0) cudaEventRecord(di.ev0[slot], st);
-    if (di.pipe_stages >= 2) kPassKernel<<<num_rows, kPassThreads, smem_pass, st>>>(P);
-    if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
-    Params R = P;
-    R.cap_s = 0;
-    if (di.pipe_stages >= 3) kRefineKernel<<<num_rows, kRefineThreads, smem_bytes_for(K, false), st>>>(R);   // + 2K words of output staging
+    // calls of more than kPipeRowsMax rows run as consecutive launches over row chunks, longest
+    // rows first, which reuse the per-row regions of the workspace
+    bool counted = false;
+    for (int hi = num_rows; hi > 0; hi -= kPipeRowsMax) {
+      P.row_end = hi;
+      P.row_begin = hi > kPipeRowsMax ? hi - kPipeRowsMax : 0;
+      const int rows = P.row_end - P.row_begin;
+      int g1 = di.sm_count * di.boundary_per_sm;
+      if (g1 > rows) g1 = rows;
+      kBoundaryKernel<<<g1, kBoundaryThreads, smem_small, st>>>(P);
+      const int slot = timing_slot(di, st);
+      if (slot >= 0) {
+        cudaEventRecord(di.ev0[slot], st);
+        if (!counted) { ++di.timed_calls; counted = true; }
+      }
+      if (di.pipe_stages >= 2) kPassKernel<<<rows, kPassThreads, smem_pass, st>>>(P);
+      if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
+      Params R = P;
+      R.cap_s = 0;
+      if (di.pipe_stages >= 3) kRefineKernel<<<rows, kRefineThreads, smem_bytes_for(K, false), st>>>(R);   // + 2K words of output staging
+    }
   } else if (di.variant == kFusedVariant) {
     const size_t fsmem = wsf::ws_smem_bytes(K, split);
     int per_sm = 0;
@@ -1886,7 +1901,7 @@ static int select_impl(const float* scores, const int32_t* row_starts, int64_t p
     // once per segment, was measured: the segments' Phase 1 run side by side anyway and the extra
     // launch is serial - config 2 went from 58 to 71 us, config 4 from 75 to 69 us.  Left out.)
     const int slot = timing_slot(di, st);
-    if (slot >= 0) cudaEventRecord(di.ev0[slot], st);
+    if (slot >= 0) { cudaEventRecord(di.ev0[slot], st); ++di.timed_calls; }
     v.fn<<<grid, v.threads, smem, st>>>(P);
     if (slot >= 0) cudaEventRecord(di.ev1[slot], st);
   }

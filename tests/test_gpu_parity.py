@@ -280,10 +280,10 @@ def test_policy_override_changes_routes_not_results():
         B.hpctopk_set_policy(100, 1.5, 1.75)            # not a power of two
 
 
-@pytest.mark.parametrize("M", [513, 8192, 8193])
+@pytest.mark.parametrize("M", [513, 8192, 8193, 17000])
 def test_many_small_rows_at_the_call_shape_limits(M):
-    """513 and 8192 rows: the smallest and the largest three-kernel call; 8193: back on the single
-    kernel.  Rows of 0..3000 scores at K=64 take the short, direct and sampled routes (the
+    """513 and 8192 rows: the smallest three-kernel call and the largest single launch of it; 8193:
+    two consecutive launches over row chunks.  Rows of 0..3000 scores at K=64 take the short, direct and sampled routes (the
     capacity at this K is 4096, so nothing here is sampled except through a longer row mixed in)."""
     K = 64
     rng = np.random.default_rng(M)
@@ -294,7 +294,7 @@ def test_many_small_rows_at_the_call_shape_limits(M):
     starts = np.concatenate([[0], np.cumsum(lengths)[:-1]]).astype(np.int32)
     batch = W.Batch(f"small_rows_{M}", scores, torch.from_numpy(starts).to(DEV),
                     torch.from_numpy(lengths.astype(np.int32)).to(DEV))
-    assert B.hpctopk_kernels_per_call(M) == (3 if M <= 8192 else 1)
+    assert B.hpctopk_kernels_per_call(M) == 3 * ((M + 8191) // 8192)
     stats, _, _, _ = _common().check_batch(batch, K, check_trace=True)
     assert stats["rows_short"] > 0 and stats["rows_direct"] > 0 and stats["rows_primary"] > 0
 
